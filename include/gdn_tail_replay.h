@@ -1,0 +1,141 @@
+/*
+ * gdn_tail_replay.h — C ABI of the B200 (sm_100a) Gated DeltaNet tail-replay library.
+ *
+ * What it computes.  For every request n and v-head h, starting from a zero state (or from
+ * desc->init_state), the Gated DeltaNet recurrence of the paper's Eq. 1 is applied to the
+ * request's rows of the packed inputs:
+ *
+ *     S_t = S_{t-1} * alpha_t * (I - beta_t k_t k_t^T) + beta_t v_t k_t^T       S in R^{dv x dk}
+ *     o_t = S_t q_t                                                            (state after token t)
+ *
+ * with alpha_t = exp(g_t), g_t = log alpha_t <= 0.  gdn_tail_replay is Eq. 2 (the recurrence
+ * restricted to the last k tokens of a matched prefix, zero start): the caller passes only the
+ * tail rows.  gdn_full_prefill is the same function over whole prefixes (the paper's
+ * full-prefill baseline).  tail_select is the replay-window arithmetic k = ceil(r m) of the
+ * paper's Method section.
+ *
+ * Layouts (row-major, packed varlen, no batch dimension; T = cu_tail_lens[N]):
+ *     q, k          [T, Hq, dk]   io_dtype (bf16 or fp32)
+ *     v             [T, Hv, dv]   io_dtype
+ *     g, beta       [T, Hv]       fp32
+ *     cu_tail_lens  [N + 1]       int32, cu[0] = 0, non-decreasing; request n owns rows
+ *                                 [cu[n], cu[n+1])
+ *     out_o         [T, Hv, dv]   io_dtype
+ *     out_state     [N, Hv, dk, dv] fp32, out_state[n,h,a,b] = S[b][a] (the transpose of S)
+ * v-head h reads q/k head h / (Hv / Hq): consecutive v-heads share one q/k head.  No scaling
+ * or normalisation is applied to q or k.  All pointers must be 16-byte aligned.
+ *
+ * Memory.  With desc->memory == GDN_MEM_DEVICE every data pointer is a device pointer.  With
+ * GDN_MEM_HOST every data pointer (q, k, v, g, beta, cu_tail_lens, out_o, out_state,
+ * init_state) is a host pointer (pinned memory makes the copies asynchronous); the library
+ * stages through the caller's workspace and copies results back on the same stream.
+ * Ownership: every buffer is the caller's.  The library allocates no device memory, keeps no
+ * state between calls and frees nothing.  Calls are asynchronous on desc->stream; buffers
+ * must stay alive until the stream has passed the call.  Valid output rows are fully
+ * overwritten; no other byte of the outputs is touched.  A request of length 0 gets a zero
+ * state (or its init_state) and no output rows.
+ *
+ * Errors.  Every function returns a gdn_status (tail_select: a length, or -1); nothing
+ * aborts or throws.  Problems visible on the host (null pointers, bad head counts,
+ * unsupported dims or chunk, workspace too small, misaligned pointers) are reported before
+ * any GPU work is enqueued.  Device data (g > 0, NaN, non-monotone cu_tail_lens on the
+ * device) is not validated.  A bounded device-side wait that expires writes
+ * GDN_ERR_TIMEOUT to *desc->status_word (if given) and the kernel returns early.
+ */
+#ifndef GDN_TAIL_REPLAY_H_
+#define GDN_TAIL_REPLAY_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#if defined(__GNUC__)
+#define GDN_API __attribute__((visibility("default")))
+#else
+#define GDN_API
+#endif
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    GDN_OK = 0,
+    GDN_ERR_INVALID_ARG = -1,   /* null / misaligned pointer, inconsistent sizes */
+    GDN_ERR_UNSUPPORTED = -2,   /* head dims, chunk, dtype or kernel choice not built */
+    GDN_ERR_WORKSPACE = -3,     /* workspace missing or smaller than gdn_workspace_size() */
+    GDN_ERR_CUDA = -4,          /* a CUDA runtime / driver call failed */
+    GDN_ERR_TIMEOUT = -5        /* device-side bounded wait expired (status_word only) */
+} gdn_status;
+
+typedef enum { GDN_F32 = 0, GDN_BF16 = 1 } gdn_dtype;
+typedef enum { GDN_MEM_DEVICE = 0, GDN_MEM_HOST = 1 } gdn_memory;
+
+/* Which kernel family runs the recurrence. */
+typedef enum {
+    GDN_KERNEL_AUTO = 0,        /* tensor-core path when the shape allows it, else the fp32 path */
+    GDN_KERNEL_FP32_SIMT = 1,   /* token-recurrent, all-fp32 FFMA; any supported shape and dtype */
+    GDN_KERNEL_TCGEN05 = 2      /* chunkwise WY form on tcgen05/TMEM; bf16, dk = dv = 128, chunk 64 */
+} gdn_kernel;
+
+typedef struct gdn_desc {
+    int32_t  num_qk_heads;      /* Hq */
+    int32_t  num_v_heads;       /* Hv, a multiple of Hq */
+    int32_t  head_k_dim;        /* dk: 64 or 128 */
+    int32_t  head_v_dim;        /* dv: 64 or 128 */
+    int32_t  io_dtype;          /* gdn_dtype of q, k, v, out_o */
+    int32_t  num_seqs;          /* N */
+    int64_t  total_tokens;      /* T = cu_tail_lens[N]; known to the caller, so no device sync */
+    int32_t  memory;            /* gdn_memory */
+    int32_t  kernel;            /* gdn_kernel */
+    const float* init_state;    /* optional [N, Hv, dk, dv] fp32 start state; NULL = zero (Eq. 2) */
+    void*    workspace;         /* caller-owned device scratch, 256-byte aligned */
+    size_t   workspace_bytes;   /* >= gdn_workspace_size(desc) */
+    int32_t* status_word;       /* optional device int32; written only on a device-side error */
+    void*    stream;            /* cudaStream_t (NULL = the legacy default stream) */
+} gdn_desc;
+
+/*
+ * Device scratch the two forward calls need for this descriptor (scheduler work list and
+ * counter; plus staging for every input and output when desc->memory == GDN_MEM_HOST).
+ * Returns 0 for an invalid descriptor.  Host-only; no CUDA call.
+ */
+GDN_API size_t gdn_workspace_size(const gdn_desc* desc);
+
+/*
+ * Tail replay (paper Eq. 2): rebuild each request's per-head state by running Eq. 1 over its
+ * tail rows from a zero state, returning o_t for every tail token and the final state.
+ * `chunk` is the chunk length of the chunkwise evaluation; the result does not depend on it
+ * mathematically; 64 is the supported value.  out_o may be NULL to skip the outputs (state
+ * rebuild only); out_state may be NULL to skip the states.
+ */
+GDN_API int32_t gdn_tail_replay(const gdn_desc* desc, const void* q, const void* k, const void* v,
+                        const float* g, const float* beta, const int32_t* cu_tail_lens,
+                        int32_t chunk, void* out_o, float* out_state);
+
+/*
+ * Full prefill (paper Eq. 1 over the whole matched prefix; the paper's "full" baseline):
+ * same arguments and semantics, cu_tail_lens holding whole prefix lengths.
+ */
+GDN_API int32_t gdn_full_prefill(const gdn_desc* desc, const void* q, const void* k, const void* v,
+                         const float* g, const float* beta, const int32_t* cu_tail_lens,
+                         int32_t chunk, void* out_o, float* out_state);
+
+/*
+ * Replay-window length k = ceil(budget_frac * prefix_len) (paper, Method section); the
+ * window is rows [prefix_len - k, prefix_len).  Clamped to [0, prefix_len]; budget_frac >= 1
+ * selects the whole prefix.  A product that is an integer mathematically but lands just above
+ * it in binary64 (0.07 * 100) is not rounded up.  Returns -1 if prefix_len < 0,
+ * budget_frac < 0 or budget_frac is NaN.  Host-only.
+ */
+GDN_API int64_t tail_select(int64_t prefix_len, double budget_frac);
+
+/* Static, human-readable text for a gdn_status value. */
+GDN_API const char* gdn_status_string(int32_t status);
+
+/* Number of kernels the last forward call on this thread enqueued (for launch accounting). */
+GDN_API int32_t gdn_last_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* GDN_TAIL_REPLAY_H_ */

@@ -1,0 +1,45 @@
+// Shared declarations of the GDN tail-replay CUDA library (host + device).
+#pragma once
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+#include "gdn_tail_replay.h"
+
+namespace gdn {
+
+// Device-side view of one forward call; all pointers are device pointers.
+struct Problem {
+    const void* q;            // [T, Hq, dk] io dtype
+    const void* k;            // [T, Hq, dk]
+    const void* v;            // [T, Hv, dv]
+    const float* g;           // [T, Hv]  log-decay
+    const float* beta;        // [T, Hv]
+    const int32_t* cu;        // [N + 1]
+    const float* init_state;  // [N, Hv, dk, dv] or nullptr
+    void* out_o;              // [T, Hv, dv] io dtype or nullptr
+    float* out_state;         // [N, Hv, dk, dv] or nullptr
+    int32_t* status_word;     // optional device int32
+    int32_t num_seqs, Hq, Hv, dk, dv;
+    int64_t total_tokens;
+};
+
+// Scheduler scratch at the head of the workspace.
+struct SchedHeader {
+    uint32_t next_item;       // dynamic work counter, reset by the scheduler kernel
+    uint32_t pad[63];
+};
+static_assert(sizeof(SchedHeader) == 256, "header is one 256-byte line");
+
+// Work list: requests ordered longest-first (paper is silent on scheduling; ragged tails from
+// concurrent cache hits differ up to 8x in length, so long chains must start first).
+struct Sched {
+    SchedHeader* header;
+    int32_t* order;           // [N] request indices, longest first
+};
+
+cudaError_t launch_scheduler(const int32_t* cu, int32_t num_seqs, const Sched& s, cudaStream_t stream);
+cudaError_t launch_simt(const Problem& p, const Sched& s, int io_dtype, cudaStream_t stream, int* launches);
+// Returns cudaErrorNotSupported when the tensor-core path cannot run this problem.
+cudaError_t launch_tcgen05(const Problem& p, const Sched& s, cudaStream_t stream, int* launches);
+
+}  // namespace gdn
