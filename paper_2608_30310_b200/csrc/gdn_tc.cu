@@ -2,22 +2,33 @@
 // tcgen05 MMAs with TMEM accumulators and TMA-staged bf16 tiles.  bf16 io, dk = dv = 128, chunk 64.
 //
 // Everything is kept in the transposed orientation so that every MMA has M = 128 (one TMEM lane
-// per value-dimension index i, or per key-dimension index for W): the carried state is
+// per value-dimension index i, or per key-dimension index for W^T): the carried state is
 // S (dv x dk, fp32, TMEM-resident), and per chunk of C = 64 tokens with start state S0:
 //
 //   G_t   = cumsum(g) inside the chunk;  Gam[t,s] = exp(G_t - G_s) (t >= s)
 //   Gram  = [K;Q] K^T                        (MMA, 128 x 64: rows 0-63 K K^T, rows 64-127 Q K^T)
 //   A     = strict_lower(beta_t Gam (K K^T)),  P = lower_incl(Gam (Q K^T))
-//   X     = (I + A)^-1                        (fp32, shared memory, blocked forward substitution)
+//   X     = (I + A)^-1                        (16 x 16 diagonal blocks by substitution in fp32, block
+//                                              merges on mma.sync tf32)
 //   T'    = X diag(beta),  T'' = X diag(beta e^G)
 //   W^T   = K^T T''^T                         (MMA, 128(dk) x 64)
 //   Dl^T  = V^T T'^T - S0 W^T                 (two MMAs into one accumulator, second negated)
 //   O^T   = (S0 Q^T) diag(e^G) + Dl^T P^T     (two MMAs, combined in the epilogue)
 //   S     = e^{G_C} S0 + (Dl diag(e^{G_C - G}))^T K    (MMA accumulating onto the pre-scaled state)
 //
-// One CTA walks one chain (request, v-head) at a time, chains handed out longest-first through an
-// atomic counter.  Padding rows of a ragged last chunk get g = 0 and beta = 0, which makes them
-// inert (their rows of A, W, U and Delta vanish); their outputs are not stored.
+// The CTA is warp-specialised and software-pipelined over the chunks of all chains it owns:
+//   warp 0      TMA producer: K/Q tiles two chunks ahead (3 slots), V one chunk ahead (1 slot)
+//   warp 1      issues the chain MMAs (U^T, S0 W^T, S0 Q^T, Dl^T P^T, state update)
+//   warp 2      issues the intra-chunk MMAs (Gram, W^T) for the next chunk
+//   warps 4-11  "pre" group: decay scan, A / P, triangular solve, T', T'', W^T epilogue (chunk j+1)
+//   warps 12-19 "chain" group: Delta epilogue, state conversion, output epilogue (chunk j)
+// Each group has two warps per TMEM lane window (they split the columns), and every per-chunk loop is
+// kept rolled with 16-column TMEM accesses: straight-line code larger than the instruction caches runs
+// at a fraction of the issue rate, so the static footprint matters as much as the instruction count.
+// Chains (request, v-head) are ordered longest-first by the scheduler kernel and dealt to CTAs in
+// snake order, so each role can walk its CTA's chunk sequence without any broadcast.  Padding rows
+// of a ragged last chunk get g = 0 and beta = 0, which makes them inert; their outputs are not stored.
+// Every mbarrier wait is bounded: on expiry the CTA records GDN_ERR_TIMEOUT and unwinds.
 #include <cuda.h>
 #include "common.cuh"
 #include "ptx.cuh"
@@ -27,30 +38,44 @@ namespace {
 
 using namespace ptx;
 
-constexpr int LDF = 68;                       // fp32 row stride of the A / X scratch (floats)
+constexpr int LDA = 68;                       // fp32 row stride of the A scratch (floats)
+constexpr int LDX = 72;                       // fp32 row stride of the X scratch
+constexpr int LDM = 40;                       // fp32 row stride of the merge scratch
 constexpr float kLog2e = 1.4426950408889634f;
+constexpr int kThreads = 640;      // 3 single-lane role warps (+1 idle), 8 pre warps, 8 chain warps
+constexpr int kWgThreads = 256;
 
 // ---- shared memory map (bytes from a 1024-aligned base) ---------------------------------------
-constexpr uint32_t SM_KQ = 0;                 // 2 halves x [128 rows: K 0-63, Q 64-127] x 128 B   32 KB
-constexpr uint32_t SM_V = 32768;              // 2 halves x [64 rows] x 128 B                       16 KB
-constexpr uint32_t SM_W = 49152;              // W [t][dk] bf16, 2 halves x 64 rows x 128 B         16 KB
-constexpr uint32_t SM_TP = 65536;             // T'  [t][s] bf16                                     8 KB
-constexpr uint32_t SM_TPP = 73728;            // T'' [t][s] bf16                                     8 KB
-constexpr uint32_t SM_P = 81920;              // P   [t][s] bf16                                     8 KB
-constexpr uint32_t SM_AF = 90112;             // A fp32 [64][LDF]
-constexpr uint32_t SM_XF = SM_AF + 64 * LDF * 4;   // X fp32 [64][LDF]
-constexpr uint32_t SM_MF = SM_XF + 64 * LDF * 4;   // 16 x 64 fp32 scratch of the blocked solve
-constexpr uint32_t SM_MISC = SM_MF + 16 * 64 * 4;
-constexpr uint32_t SM_TOTAL = SM_MISC + 2048;
-constexpr uint32_t SMEM_BYTES = SM_TOTAL + 1024;   // slack for the manual 1024-byte alignment
+constexpr uint32_t SM_KQ = 0;                 // 3 slots x {2 halves x [128 rows: K 0-63, Q 64-127] x 128 B}  96 KB
+constexpr uint32_t KQ_SLOT = 32768;
+constexpr uint32_t SM_V = 98304;              // 2 halves x [64 rows] x 128 B                               16 KB
+constexpr uint32_t SM_WT = 114688;            // W^T [dk][t] bf16, 128 rows x 128 B                          16 KB
+constexpr uint32_t SM_TP = 131072;            // T'  [t][s] bf16                                             8 KB
+constexpr uint32_t SM_TPP = 139264;           // T'' [t][s] bf16                                             8 KB
+constexpr uint32_t SM_P = 147456;             // 2 x P [t][s] bf16                                          16 KB
+constexpr uint32_t SM_OST = 163840;           // O staging [t][dv] bf16                                     16 KB
+constexpr uint32_t SM_AF = 180224;            // A fp32 [64][LDA]
+constexpr uint32_t SM_XF = SM_AF + 64 * LDA * 4;   // X fp32 [64][LDX]
+constexpr uint32_t SM_MF = SM_XF + 64 * LDX * 4;   // merge scratch fp32 [32][LDM]
+constexpr uint32_t SM_MISC = SM_MF + 32 * LDM * 4;
 
-struct Misc {
-    float g[64], beta[64], G[64], eG[64], eRest[64];
-    unsigned long long bar_tma, bar_mma;
-    uint32_t tmem_base, item, abort;
-    float eGC;
+enum Bar {
+    B_FULL_KQ0 = 0, B_FULL_KQ1, B_FULL_KQ2, B_FULL_V, B_GRAM_DONE, B_W_DONE, B_U_DONE, B_MMA1_DONE,
+    B_MMA3_DONE, B_KQ_FREE0, B_KQ_FREE1, B_KQ_FREE2, B_P_FREE0, B_P_FREE1, B_WACC_READ, B_TPP_READY,
+    B_PRE_DONE0, B_PRE_DONE1, B_D_READY, B_SBF_READY, B_ACC23_FREE, NUM_BARS
 };
-static_assert(sizeof(Misc) <= 2048, "misc block");
+
+// G2 = log2(e) * cumulative log-decay; bE = beta e^G; eG = e^G; eRest = e^{G_C - G}
+struct Decay { float G2[64], beta[64], bE[64], eG[64], eRest[64]; };
+struct Misc {
+    Decay decay[4];                    // per-chunk decay factors, ring of 4 (pre writes, chain reads)
+    unsigned long long bars[NUM_BARS];
+    uint32_t tmem_base;
+    volatile uint32_t abort;
+};
+constexpr uint32_t SM_TOTAL = SM_MISC + ((sizeof(Misc) + 1023) / 1024) * 1024;
+constexpr uint32_t SMEM_BYTES = SM_TOTAL + 1024;   // slack for the manual 1024-byte alignment
+static_assert(SMEM_BYTES <= 232448, "exceeds the 227 KB shared memory of one CTA");
 
 // ---- TMEM column map (512 columns x 128 lanes x 32 bit) ----------------------------------------
 constexpr uint32_t TM_S32 = 0;      // fp32 state S (dv x dk), 128 columns
@@ -58,13 +83,13 @@ constexpr uint32_t TM_SBF = 128;    // bf16 copy of the chunk-start state, 64 co
 constexpr uint32_t TM_ACC1 = 192;   // Delta^T accumulator (U^T - S0 W^T), 64 columns
 constexpr uint32_t TM_ACC2 = 256;   // S0 Q^T, 64 columns
 constexpr uint32_t TM_ACC3 = 320;   // Delta^T P^T, 64 columns
-constexpr uint32_t TM_DBF = 384;    // Delta^T bf16, 32 columns
-constexpr uint32_t TM_DPBF = 416;   // (Delta diag(e^{G_C - G}))^T bf16, 32 columns
-constexpr uint32_t TM_GRAM = 448;   // Gram accumulator, later W^T accumulator, 64 columns
+constexpr uint32_t TM_GRAM = 384;   // Gram accumulator, later W^T accumulator, 64 columns
+constexpr uint32_t TM_DBF = 448;    // Delta^T bf16, 32 columns
+constexpr uint32_t TM_DPBF = 480;   // (Delta diag(e^{G_C - G}))^T bf16, 32 columns
 
 constexpr uint32_t ID_GRAM = idesc_bf16(128, 64, 0, 0, 0);    // [K;Q] (K-major) x K (K-major)
 constexpr uint32_t ID_WU = idesc_bf16(128, 64, 1, 0, 0);      // K^T or V^T (M-major) x T (K-major)
-constexpr uint32_t ID_SW = idesc_bf16(128, 64, 0, 0, 1);      // -S0 (TMEM) x W (K-major)
+constexpr uint32_t ID_SW = idesc_bf16(128, 64, 0, 1, 1);      // -S0 (TMEM) x W^T (N-major)
 constexpr uint32_t ID_SQ = idesc_bf16(128, 64, 0, 0, 0);      // S0 (TMEM) x Q (K-major)
 constexpr uint32_t ID_DP = idesc_bf16(128, 64, 0, 0, 0);      // Delta^T (TMEM) x P (K-major)
 constexpr uint32_t ID_DK = idesc_bf16(128, 128, 0, 1, 0);     // Delta'^T (TMEM) x K (N-major)
@@ -77,441 +102,741 @@ struct TcParams {
 
 #ifdef GDN_TC_DEBUG
 constexpr int DBG_STRIDE = 61440;
+#define GDN_DBG(x) x
+#define GDN_T(i) do { long long n_ = clock64(); tt_[i] += n_ - tl_; tl_ = n_; } while (0)
+#else
+#define GDN_DBG(x)
+#define GDN_T(i) do {} while (0)
 #endif
 
-__global__ void __launch_bounds__(128, 1)
+// Walks the chunk sequence of one CTA: chains dealt in snake order over the longest-first list,
+// chunks of 64 rows inside each chain.  Every role keeps its own cursor(s).
+struct ChunkCursor {
+    const Problem* p;
+    const int32_t* order;
+    int r, n, h, hq, row_begin, row_end, nchunks, c;
+    uint32_t num_items;
+    bool valid;
+
+    __device__ void init(const Problem* pp, const int32_t* ord)
+    {
+        p = pp; order = ord; r = -1; c = 0; nchunks = 0; valid = true;
+        num_items = (uint32_t)pp->num_seqs * (uint32_t)pp->Hv;
+        next_chain();
+    }
+    __device__ static uint32_t item_of(int round)
+    {
+        const uint32_t G = gridDim.x, b = blockIdx.x;
+        return (uint32_t)round * G + ((round & 1) ? (G - 1 - b) : b);
+    }
+    // moves to the next chain that has at least one chunk
+    __device__ void next_chain()
+    {
+        for (;;) {
+            ++r;
+            const uint32_t item = item_of(r);
+            if (item >= num_items) { valid = false; return; }
+            n = order[item / p->Hv];
+            h = item % p->Hv;
+            hq = h / (p->Hv / p->Hq);
+            row_begin = p->cu[n];
+            row_end = p->cu[n + 1];
+            nchunks = (row_end - row_begin + 63) >> 6;
+            c = 0;
+            if (nchunks > 0) return;
+        }
+    }
+    __device__ void advance()
+    {
+        if (++c >= nchunks) next_chain();
+    }
+    __device__ int row0() const { return row_begin + c * 64; }
+    __device__ int nvalid() const { return min(64, row_end - row0()); }
+    __device__ bool first() const { return c == 0; }
+    __device__ bool last() const { return c == nchunks - 1; }
+};
+
+struct Ctx {
+    uint32_t sb;          // shared-space address of the aligned base
+    uint8_t* sm;          // generic pointer to the same place
+    Misc* misc;
+    uint32_t tmem;
+    __device__ uint32_t bar(int i) const { return sb + SM_MISC + (uint32_t)offsetof(Misc, bars) + 8u * i; }
+    // Bounded wait.  On expiry it raises the CTA-wide abort flag; from then on no wait blocks any more, so
+    // every role still runs through its (data-independent) loop structure, keeps meeting its warpgroup
+    // barriers and reaches the end of the kernel; the results are garbage and the host sees the status word.
+    __device__ bool wait(int i, uint32_t parity) const
+    {
+        const uint32_t b = bar(i);
+        if (mbar_try_wait(b, parity)) return true;
+        if (misc->abort) return true;
+        const uint64_t t0 = globaltimer_ns();
+        for (uint32_t it = 0;; ++it) {
+            __nanosleep(40);                       // back off: spinning warps would steal issue slots
+            if (mbar_try_wait(b, parity)) return true;
+            if ((it & 63u) == 63u) {
+                if (misc->abort) return true;
+                if (globaltimer_ns() - t0 > 2000000000ull) { misc->abort = 1u; return true; }
+            }
+        }
+    }
+};
+
+__device__ __forceinline__ void wg_sync(int id) { asm volatile("bar.sync %0, 256;" ::"r"(id) : "memory"); }
+__device__ __forceinline__ uint32_t to_tf32(float x)
+{
+    uint32_t r;
+    asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(r) : "f"(x));
+    return r;
+}
+__device__ __forceinline__ void mma_tf32(float (&c)[4], const uint32_t (&a)[4], const uint32_t (&b)[2])
+{
+    asm volatile("mma.sync.aligned.m16n8k8.row.col.f32.tf32.tf32.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                 : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+                 : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b[0]), "r"(b[1]));
+}
+// 16 x 8 tile of C += A[r0.., k0..k1) * B[k0..k1, n0..): A, B row-major fp32 (tf32-rounded) in shared memory
+__device__ __forceinline__ void tile_mma(float (&c)[4], const float* A, int lda, int r0, const float* B, int ldb,
+                                         int n0, int k0, int k1, int lane)
+{
+    const int g = lane >> 2, t4 = lane & 3;
+    for (int k = k0; k < k1; k += 8) {
+        uint32_t a[4], b[2];
+        a[0] = __float_as_uint(A[(r0 + g) * lda + k + t4]);
+        a[1] = __float_as_uint(A[(r0 + g + 8) * lda + k + t4]);
+        a[2] = __float_as_uint(A[(r0 + g) * lda + k + t4 + 4]);
+        a[3] = __float_as_uint(A[(r0 + g + 8) * lda + k + t4 + 4]);
+        b[0] = __float_as_uint(B[(k + t4) * ldb + n0 + g]);
+        b[1] = __float_as_uint(B[(k + t4 + 4) * ldb + n0 + g]);
+        mma_tf32(c, a, b);
+    }
+}
+// stores a 16 x 8 C tile (optionally negated), rounded to tf32, at D[r0.., n0..)
+__device__ __forceinline__ void tile_store(const float (&c)[4], float sign, float* D, int ldd, int r0, int n0, int lane)
+{
+    const int g = lane >> 2, t4 = lane & 3;
+    float2 lo = make_float2(__uint_as_float(to_tf32(sign * c[0])), __uint_as_float(to_tf32(sign * c[1])));
+    float2 hi = make_float2(__uint_as_float(to_tf32(sign * c[2])), __uint_as_float(to_tf32(sign * c[3])));
+    *reinterpret_cast<float2*>(&D[(r0 + g) * ldd + n0 + 2 * t4]) = lo;
+    *reinterpret_cast<float2*>(&D[(r0 + g + 8) * ldd + n0 + 2 * t4]) = hi;
+}
+
+// ================================================================================================
+// warp 0: TMA producer
+// ================================================================================================
+__device__ void role_producer(const Ctx& cx, const TcParams& prm, const CUtensorMap* tm_q, const CUtensorMap* tm_k,
+                              const CUtensorMap* tm_v)
+{
+    ChunkCursor ckq, cv;                 // K/Q runs two chunks ahead of V
+    ckq.init(&prm.p, prm.s.order);
+    cv = ckq;
+    auto load_kq = [&](const ChunkCursor& cc, uint32_t j) {
+        const uint32_t slot = j % 3u, dst = cx.sb + SM_KQ + slot * KQ_SLOT, bar = cx.bar(B_FULL_KQ0 + slot);
+        mbar_arrive_expect_tx(bar, 32768u);
+        tma_load_2d(dst, tm_k, cc.hq * 128, cc.row0(), bar);
+        tma_load_2d(dst + 16384, tm_k, cc.hq * 128 + 64, cc.row0(), bar);
+        tma_load_2d(dst + 8192, tm_q, cc.hq * 128, cc.row0(), bar);
+        tma_load_2d(dst + 24576, tm_q, cc.hq * 128 + 64, cc.row0(), bar);
+    };
+    uint32_t jkq = 0;
+    for (; jkq < 2 && ckq.valid; ++jkq) { load_kq(ckq, jkq); ckq.advance(); }
+#pragma unroll 1
+    for (uint32_t j = 0; cv.valid; ++j) {
+        // V(j): the single slot is free once U^T MMA of chunk j-1 has completed
+        if (j >= 1) cx.wait(B_U_DONE, (j - 1) & 1u);
+        const uint32_t bar = cx.bar(B_FULL_V);
+        mbar_arrive_expect_tx(bar, 16384u);
+        tma_load_2d(cx.sb + SM_V, tm_v, cv.h * 128, cv.row0(), bar);
+        tma_load_2d(cx.sb + SM_V + 8192, tm_v, cv.h * 128 + 64, cv.row0(), bar);
+        cv.advance();
+        // K/Q(j+2): its slot held chunk j-1, free once the state-update MMA of chunk j-1 has completed
+        if (ckq.valid) {
+            if (jkq >= 3) cx.wait(B_KQ_FREE0 + jkq % 3u, ((jkq / 3u) - 1u) & 1u);
+            load_kq(ckq, jkq);
+            ckq.advance();
+            ++jkq;
+        }
+    }
+}
+
+// advances the start-address field of a shared-memory descriptor by a byte offset
+__device__ __forceinline__ uint64_t desc_add(uint64_t d, uint32_t bytes) { return d + (uint64_t)(bytes >> 4); }
+
+// ================================================================================================
+// warp 2: intra-chunk MMAs (Gram and W^T) for the chunk the pre group works on
+// ================================================================================================
+__device__ void role_mma_pre(const Ctx& cx, const TcParams& prm)
+{
+    ChunkCursor cc;
+    cc.init(&prm.p, prm.s.order);
+    const uint64_t d_tpp = smem_desc_sw128(cx.sb + SM_TPP, 16, 1024);
+#pragma unroll 1
+    for (uint32_t j = 0; cc.valid; ++j, cc.advance()) {
+        const uint32_t slot = j % 3u, kq = cx.sb + SM_KQ + slot * KQ_SLOT;
+        const uint64_t d_kq = smem_desc_sw128(kq, 16, 1024);            // [K;Q] rows, K-major
+        const uint64_t d_kt = smem_desc_sw128(kq, 16384, 1024);         // K tile as M-major operand (K^T)
+        cx.wait(B_FULL_KQ0 + slot, (j / 3u) & 1u);
+        if (j >= 1) cx.wait(B_WACC_READ, (j - 1) & 1u);
+        tc_fence_after();
+#pragma unroll 1
+        for (int ks = 0; ks < 8; ++ks) {
+            const uint64_t d = desc_add(d_kq, (ks >> 2) * 16384 + (ks & 3) * 32);
+            mma_ss(cx.tmem + TM_GRAM, d, d, ID_GRAM, ks > 0);
+        }
+        mma_commit(cx.bar(B_GRAM_DONE));
+        cx.wait(B_TPP_READY, j & 1u);
+        tc_fence_after();
+#pragma unroll 1
+        for (int ks = 0; ks < 4; ++ks)
+            mma_ss(cx.tmem + TM_GRAM, desc_add(d_kt, ks * 2048), desc_add(d_tpp, ks * 32), ID_WU, ks > 0);
+        mma_commit(cx.bar(B_W_DONE));
+    }
+}
+
+// ================================================================================================
+// warp 1: chain MMAs
+// ================================================================================================
+__device__ void role_mma_chain(const Ctx& cx, const TcParams& prm)
+{
+    ChunkCursor cc;
+    cc.init(&prm.p, prm.s.order);
+    const uint64_t d_v = smem_desc_sw128(cx.sb + SM_V, 8192, 1024);     // V tile as M-major operand (V^T)
+    const uint64_t d_tp = smem_desc_sw128(cx.sb + SM_TP, 16, 1024);
+    const uint64_t d_wt = smem_desc_sw128(cx.sb + SM_WT, 16, 1024);     // W^T rows [dk][t], N-major operand
+#pragma unroll 1
+    for (uint32_t j = 0; cc.valid; ++j, cc.advance()) {
+        const uint32_t kq = cx.sb + SM_KQ + (j % 3u) * KQ_SLOT;
+        const uint64_t d_q = smem_desc_sw128(kq + 8192, 16, 1024);      // Q rows, K-major
+        const uint64_t d_kn = smem_desc_sw128(kq, 16384, 1024);         // K tile as N-major operand
+        const uint64_t d_p = smem_desc_sw128(cx.sb + SM_P + (j & 1u) * 8192, 16, 1024);
+        const bool first = cc.first();
+        cx.wait(B_PRE_DONE0 + (j & 1u), (j >> 1) & 1u);
+        cx.wait(B_FULL_V, j & 1u);
+        tc_fence_after();
+        // U^T = V^T T'^T -> ACC1 (free: the Delta epilogue of chunk j-1 came before that chunk's last MMAs)
+#pragma unroll 1
+        for (int ks = 0; ks < 4; ++ks)
+            mma_ss(cx.tmem + TM_ACC1, desc_add(d_v, ks * 2048), desc_add(d_tp, ks * 32), ID_WU, ks > 0);
+        mma_commit(cx.bar(B_U_DONE));
+        // state of the previous chunk converted (or, at a chain start, the previous chain's state read out)
+        if (j >= 1) cx.wait(B_SBF_READY, (j - 1) & 1u);
+        tc_fence_after();
+        if (!first) {
+#pragma unroll 1
+            for (int ks = 0; ks < 8; ++ks)
+                mma_ts(cx.tmem + TM_ACC1, cx.tmem + TM_SBF + ks * 8, desc_add(d_wt, ks * 2048), ID_SW, 1u);
+        }
+        if (j >= 1) cx.wait(B_ACC23_FREE, (j - 1) & 1u);
+        tc_fence_after();
+        if (!first) {
+#pragma unroll 1
+            for (int ks = 0; ks < 8; ++ks)
+                mma_ts(cx.tmem + TM_ACC2, cx.tmem + TM_SBF + ks * 8,
+                       desc_add(d_q, (ks >> 2) * 16384 + (ks & 3) * 32), ID_SQ, ks > 0);
+        }
+        mma_commit(cx.bar(B_MMA1_DONE));
+        cx.wait(B_D_READY, j & 1u);
+        tc_fence_after();
+#pragma unroll 1
+        for (int ks = 0; ks < 4; ++ks)
+            mma_ts(cx.tmem + TM_ACC3, cx.tmem + TM_DBF + ks * 8, desc_add(d_p, ks * 32), ID_DP, ks > 0);
+#pragma unroll 1
+        for (int ks = 0; ks < 4; ++ks)
+            mma_ts(cx.tmem + TM_S32, cx.tmem + TM_DPBF + ks * 8, desc_add(d_kn, ks * 2048), ID_DK,
+                   (!first || ks > 0) ? 1u : 0u);
+        mma_commit(cx.bar(B_MMA3_DONE));
+        mma_commit(cx.bar(B_KQ_FREE0 + j % 3u));
+        mma_commit(cx.bar(B_P_FREE0 + (j & 1u)));
+    }
+}
+
+// ================================================================================================
+// warps 4-11: pre group (intra-chunk stage of the chunk one ahead of the chain)
+// ================================================================================================
+__device__ void role_pre(const Ctx& cx, const TcParams& prm, int wtid)
+{
+    const Problem& p = prm.p;
+    const int lane = wtid & 31, pw = wtid >> 5;          // pw = 0..7
+    const int w4 = pw & 3, hf = pw >> 2;                 // TMEM lane window, column half
+    const uint32_t tl = cx.tmem + ((uint32_t)(w4 * 32) << 16);
+    float* AF = reinterpret_cast<float*>(cx.sm + SM_AF);
+    float* XF = reinterpret_cast<float*>(cx.sm + SM_XF);
+    float* MF = reinterpret_cast<float*>(cx.sm + SM_MF);
+    Misc* misc = cx.misc;
+    ChunkCursor cc;
+    cc.init(&p, prm.s.order);
+    GDN_DBG(long long tt_[16] = {0}; long long tl_ = clock64(); int nch = 0;)
+#pragma unroll 1
+    for (uint32_t j = 0; cc.valid; ++j, cc.advance()) {
+        const int row0 = cc.row0(), nvalid = cc.nvalid(), h = cc.h;
+        Decay& dc = misc->decay[j & 3u];
+        GDN_DBG(const bool dbg = prm.debug && blockIdx.x == 0 && cc.r == 0 && cc.c < 2;
+                float* dbase = prm.debug + cc.c * DBG_STRIDE;)
+
+        // ---- decay scan: every warp scans the 64 log-decays (two per lane); warp 0 publishes ------------
+        const bool ok0 = lane < nvalid, ok1 = lane + 32 < nvalid;
+        const float g0 = ok0 ? p.g[(size_t)(row0 + lane) * p.Hv + h] : 0.f;
+        const float g1 = ok1 ? p.g[(size_t)(row0 + lane + 32) * p.Hv + h] : 0.f;
+        const float b0 = ok0 ? p.beta[(size_t)(row0 + lane) * p.Hv + h] : 0.f;
+        const float b1 = ok1 ? p.beta[(size_t)(row0 + lane + 32) * p.Hv + h] : 0.f;
+        float G0 = g0 * kLog2e, G1 = g1 * kLog2e;
+#pragma unroll
+        for (int off = 1; off < 32; off <<= 1) {
+            const float u0 = __shfl_up_sync(0xffffffffu, G0, off), u1 = __shfl_up_sync(0xffffffffu, G1, off);
+            if (lane >= off) { G0 += u0; G1 += u1; }
+        }
+        G1 += __shfl_sync(0xffffffffu, G0, 31);
+        if (pw == 0) {
+            const float GC = __shfl_sync(0xffffffffu, G1, 31);
+            const float e0 = ex2_approx(G0), e1 = ex2_approx(G1);
+            dc.G2[lane] = G0; dc.G2[lane + 32] = G1;
+            dc.beta[lane] = b0; dc.beta[lane + 32] = b1;
+            dc.bE[lane] = b0 * e0; dc.bE[lane + 32] = b1 * e1;
+            dc.eG[lane] = e0; dc.eG[lane + 32] = e1;
+            dc.eRest[lane] = ex2_approx(GC - G0); dc.eRest[lane + 32] = ex2_approx(GC - G1);
+        }
+        // this thread's row of the Gram tile: lane windows 0,1 hold K K^T rows, 2,3 hold Q K^T rows
+        const int t = ((w4 & 1) << 5) + lane;
+        const bool isA = w4 < 2;
+        const float G2t = (w4 & 1) ? G1 : G0;
+        const float rowscale = isA ? ((w4 & 1) ? b1 : b0) : 1.f;
+        const int t_lim = isA ? t : t + 1;               // keep columns s < t_lim
+        wg_sync(1);                                       // decay arrays visible
+        GDN_T(0);
+
+        // ---- Gram tile -> A (fp32 scratch) and P (bf16 operand), 16 columns at a time ----------------------
+        cx.wait(B_GRAM_DONE, j & 1u);
+        GDN_T(1);
+        tc_fence_after();
+        // the P buffer of chunk j was last read by the MMAs of chunk j-2
+        if (j >= 2) cx.wait(B_P_FREE0 + (j & 1u), ((j >> 1) - 1u) & 1u);
+        {
+            uint8_t* prow = cx.sm + SM_P + (j & 1u) * 8192 + t * 128;
+#pragma unroll 1
+            for (int g = 0; g < 2; ++g) {
+                const int cb = 2 * hf + g, c0 = 16 * cb;
+                if (c0 > ((w4 & 1) << 5) + 31) {          // block entirely above the diagonal (warp-uniform)
+                    if (!isA) {
+                        *reinterpret_cast<uint4*>(prow + (((2 * cb) ^ (t & 7)) << 4)) = make_uint4(0u, 0u, 0u, 0u);
+                        *reinterpret_cast<uint4*>(prow + (((2 * cb + 1) ^ (t & 7)) << 4)) = make_uint4(0u, 0u, 0u, 0u);
+                    }
+                    continue;
+                }
+                uint32_t acc[16];
+                tmem_ld16(tl + TM_GRAM + c0, acc);
+                tmem_ld_wait();
+#ifdef GDN_TC_DEBUG
+                if (dbg) {
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) dbase[(w4 * 32 + lane) * 64 + c0 + i] = __uint_as_float(acc[i]);
+                }
+#endif
+                float vals[16];
+#pragma unroll
+                for (int i4 = 0; i4 < 4; ++i4) {
+                    const float4 gs = *reinterpret_cast<const float4*>(&dc.G2[c0 + 4 * i4]);
+                    const float gss[4] = {gs.x, gs.y, gs.z, gs.w};
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        const int i = 4 * i4 + e;
+                        const float f = ex2_approx(fminf(G2t - gss[e], 0.f)) * rowscale;
+                        vals[i] = (c0 + i < t_lim) ? f * __uint_as_float(acc[i]) : 0.f;
+                    }
+                }
+                if (isA) {
+                    float* arow = AF + t * LDA + c0;
+#pragma unroll
+                    for (int i = 0; i < 16; i += 4)
+                        *reinterpret_cast<float4*>(arow + i) = make_float4(
+                            __uint_as_float(to_tf32(vals[i])), __uint_as_float(to_tf32(vals[i + 1])),
+                            __uint_as_float(to_tf32(vals[i + 2])), __uint_as_float(to_tf32(vals[i + 3])));
+                } else {
+#pragma unroll
+                    for (int c8 = 0; c8 < 2; ++c8) {
+                        uint4 u;
+                        u.x = pack_bf16x2(vals[c8 * 8 + 0], vals[c8 * 8 + 1]);
+                        u.y = pack_bf16x2(vals[c8 * 8 + 2], vals[c8 * 8 + 3]);
+                        u.z = pack_bf16x2(vals[c8 * 8 + 4], vals[c8 * 8 + 5]);
+                        u.w = pack_bf16x2(vals[c8 * 8 + 6], vals[c8 * 8 + 7]);
+                        *reinterpret_cast<uint4*>(prow + (((2 * cb + c8) ^ (t & 7)) << 4)) = u;
+                    }
+                }
+            }
+        }
+        tc_fence_before();
+        wg_sync(1);
+        GDN_T(2);
+
+        // ---- X = (I + A)^-1 ----------------------------------------------------------------------------
+        // level 0: the four 16 x 16 diagonal blocks by forward substitution; warps 0 and 1 take two blocks
+        // each (lane & 15 owns a column of block 2 pw + (lane >> 4))
+        if (pw < 2) {
+            const int b = (2 * pw + (lane >> 4)) * 16, jj = lane & 15;
+            float x[16];
+#pragma unroll
+            for (int r = 0; r < 16; ++r) x[r] = (r == jj) ? 1.f : 0.f;
+#pragma unroll
+            for (int r = 1; r < 16; ++r) {
+                float acc0 = 0.f, acc1 = 0.f;
+#pragma unroll
+                for (int s2 = 0; s2 + 1 < r; s2 += 2) {
+                    acc0 = fmaf(AF[(b + r) * LDA + b + s2], x[s2], acc0);
+                    acc1 = fmaf(AF[(b + r) * LDA + b + s2 + 1], x[s2 + 1], acc1);
+                }
+                if (r & 1) acc0 = fmaf(AF[(b + r) * LDA + b + r - 1], x[r - 1], acc0);
+                x[r] = (r > jj) ? -(acc0 + acc1) : x[r];
+            }
+#pragma unroll
+            for (int r = 0; r < 16; ++r) XF[(b + r) * LDX + b + jj] = __uint_as_float(to_tf32(x[r]));
+        }
+        wg_sync(1);
+        GDN_T(3);
+        // level 1: X[2p+1][2p] = -X[2p+1][2p+1] (A[2p+1][2p] X[2p][2p]); warps 0-3 -> (pair p, 8-column half)
+        {
+            const int pr = (pw >> 1) & 1, nh = pw & 1, rb = 32 * pr + 16, cb0 = 32 * pr;
+            if (pw < 4) {
+                float c4[4] = {0.f, 0.f, 0.f, 0.f};
+                tile_mma(c4, AF + cb0, LDA, rb, XF + cb0 * LDX + cb0, LDX, 8 * nh, 0, 16, lane);
+                tile_store(c4, 1.f, MF, LDM, 16 * pr, 8 * nh, lane);
+            }
+            wg_sync(1);
+            if (pw < 4) {
+                float d4[4] = {0.f, 0.f, 0.f, 0.f};
+                tile_mma(d4, XF + rb, LDX, rb, MF + 16 * pr * LDM, LDM, 8 * nh, 0, 16, lane);
+                tile_store(d4, -1.f, XF + cb0, LDX, rb, 8 * nh, lane);
+            }
+            wg_sync(1);
+        }
+        GDN_T(4);
+        // level 2: X[32:64][0:32] = -X22 (A21 X11); warp -> 16 x 8 output tile (mt, nt, nh)
+        {
+            const int mt = pw >> 2, nt = (pw >> 1) & 1, nh = pw & 1, n0 = 16 * nt + 8 * nh;
+            float c4[4] = {0.f, 0.f, 0.f, 0.f};
+            // X11 is lower triangular: columns of block nt start at row 16 nt
+            tile_mma(c4, AF, LDA, 32 + 16 * mt, XF, LDX, n0, 16 * nt, 32, lane);
+            tile_store(c4, 1.f, MF, LDM, 16 * mt, n0, lane);
+            wg_sync(1);
+            float d4[4] = {0.f, 0.f, 0.f, 0.f};
+            // X22 is lower triangular: row block mt ends at column 16 (mt + 1)
+            tile_mma(d4, XF + 32, LDX, 32 + 16 * mt, MF, LDM, n0, 0, 16 * (mt + 1), lane);
+            tile_store(d4, -1.f, XF, LDX, 32 + 16 * mt, n0, lane);
+            wg_sync(1);
+        }
+        GDN_T(5);
+#ifdef GDN_TC_DEBUG
+        if (dbg) for (int e = wtid; e < 4096; e += kWgThreads) dbase[8192 + e] = ((e & 63) <= (e >> 6)) ? XF[(e >> 6) * LDX + (e & 63)] : 0.f;
+#endif
+        // ---- T'' = X diag(beta e^G) (operand of the W^T MMA), T' = X diag(beta) (operand of the U^T MMA) ----
+        // T' is single-buffered: the U^T MMA of chunk j-1 must have read it
+        if (j >= 1) cx.wait(B_U_DONE, (j - 1) & 1u);
+        {
+            const int tt = wtid >> 2, q = wtid & 3, c0 = 16 * q;      // row, 16-column quarter
+            uint32_t w1[8], w2[8];
+#pragma unroll
+            for (int i4 = 0; i4 < 4; ++i4) {
+                const float4 xv = *reinterpret_cast<const float4*>(&XF[tt * LDX + c0 + 4 * i4]);
+                const float4 bv = *reinterpret_cast<const float4*>(&dc.beta[c0 + 4 * i4]);
+                const float4 ev = *reinterpret_cast<const float4*>(&dc.bE[c0 + 4 * i4]);
+                const int s0 = c0 + 4 * i4;
+                const float x0 = (s0 <= tt) ? xv.x : 0.f, x1 = (s0 + 1 <= tt) ? xv.y : 0.f;
+                const float x2 = (s0 + 2 <= tt) ? xv.z : 0.f, x3 = (s0 + 3 <= tt) ? xv.w : 0.f;
+                w1[2 * i4] = pack_bf16x2(x0 * bv.x, x1 * bv.y);
+                w1[2 * i4 + 1] = pack_bf16x2(x2 * bv.z, x3 * bv.w);
+                w2[2 * i4] = pack_bf16x2(x0 * ev.x, x1 * ev.y);
+                w2[2 * i4 + 1] = pack_bf16x2(x2 * ev.z, x3 * ev.w);
+            }
+            const uint32_t o0 = tt * 128 + (((2 * q) ^ (tt & 7)) << 4), o1 = tt * 128 + (((2 * q + 1) ^ (tt & 7)) << 4);
+            *reinterpret_cast<uint4*>(cx.sm + SM_TP + o0) = make_uint4(w1[0], w1[1], w1[2], w1[3]);
+            *reinterpret_cast<uint4*>(cx.sm + SM_TP + o1) = make_uint4(w1[4], w1[5], w1[6], w1[7]);
+            *reinterpret_cast<uint4*>(cx.sm + SM_TPP + o0) = make_uint4(w2[0], w2[1], w2[2], w2[3]);
+            *reinterpret_cast<uint4*>(cx.sm + SM_TPP + o1) = make_uint4(w2[4], w2[5], w2[6], w2[7]);
+        }
+        fence_proxy_async_smem();
+        mbar_arrive(cx.bar(B_TPP_READY));
+        GDN_T(6);
+
+        // ---- W^T epilogue: bf16 rows [dk][t] as the N-major operand of the S0 W^T MMA ----------------------
+        cx.wait(B_W_DONE, j & 1u);
+        GDN_T(7);
+        tc_fence_after();
+        // W^T is single-buffered: the S0 W^T MMA of chunk j-1 must have read it
+        if (j >= 1) cx.wait(B_MMA1_DONE, (j - 1) & 1u);
+        {
+            const int drow = w4 * 32 + lane;                      // dk index = TMEM lane
+            uint8_t* wrow = cx.sm + SM_WT + drow * 128;
+#pragma unroll 1
+            for (int g = 0; g < 2; ++g) {
+                const int c0 = 32 * hf + 16 * g;
+                uint32_t acc[16];
+                tmem_ld16(tl + TM_GRAM + c0, acc);
+                tmem_ld_wait();
+#ifdef GDN_TC_DEBUG
+                if (dbg) {
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) dbase[12288 + drow * 64 + c0 + i] = __uint_as_float(acc[i]);
+                }
+#endif
+#pragma unroll
+                for (int c8 = 0; c8 < 2; ++c8) {
+                    uint4 u;
+                    u.x = pack_bf16x2(__uint_as_float(acc[c8 * 8 + 0]), __uint_as_float(acc[c8 * 8 + 1]));
+                    u.y = pack_bf16x2(__uint_as_float(acc[c8 * 8 + 2]), __uint_as_float(acc[c8 * 8 + 3]));
+                    u.z = pack_bf16x2(__uint_as_float(acc[c8 * 8 + 4]), __uint_as_float(acc[c8 * 8 + 5]));
+                    u.w = pack_bf16x2(__uint_as_float(acc[c8 * 8 + 6]), __uint_as_float(acc[c8 * 8 + 7]));
+                    *reinterpret_cast<uint4*>(wrow + ((((c0 >> 3) + c8) ^ (drow & 7)) << 4)) = u;
+                }
+            }
+        }
+        tc_fence_before();
+        mbar_arrive(cx.bar(B_WACC_READ));                  // the accumulator may take the next Gram tile
+        fence_proxy_async_smem();
+        mbar_arrive(cx.bar(B_PRE_DONE0 + (j & 1u)));
+        GDN_T(8);
+        GDN_DBG(++nch;)
+    }
+#ifdef GDN_TC_DEBUG
+    if (prm.debug && blockIdx.x == 0 && wtid == 0 && nch > 0) {
+        float* d = prm.debug + 2 * DBG_STRIDE;
+        d[0] = (float)nch;
+        for (int i = 0; i < 12; ++i) d[1 + i] = (float)tt_[i] / nch;
+    }
+#endif
+}
+
+// ================================================================================================
+// warps 12-19: chain group (Delta epilogue, state conversion, outputs, final state)
+// ================================================================================================
+__device__ void role_chain(const Ctx& cx, const TcParams& prm, int wtid)
+{
+    const Problem& p = prm.p;
+    const int lane = wtid & 31, cw = wtid >> 5;
+    const int w4 = cw & 3, hf = cw >> 2;                  // TMEM lane window, column half
+    const int dv = w4 * 32 + lane;                        // value-dimension index = TMEM lane
+    const uint32_t tl = cx.tmem + ((uint32_t)(w4 * 32) << 16);
+    Misc* misc = cx.misc;
+    __nv_bfloat16* __restrict__ og = reinterpret_cast<__nv_bfloat16*>(p.out_o);
+    const uint32_t num_items = (uint32_t)p.num_seqs * (uint32_t)p.Hv;
+    GDN_DBG(long long tt_[16] = {0}; long long tl_ = clock64(); int nch = 0;)
+
+    uint32_t j = 0;
+#pragma unroll 1
+    for (int r = 0;; ++r) {
+        const uint32_t item = ChunkCursor::item_of(r);
+        if (item >= num_items) break;
+        const int n = prm.s.order[item / p.Hv];
+        const int h = item % p.Hv;
+        const int row_begin = p.cu[n], row_end = p.cu[n + 1];
+        const int nchunks = (row_end - row_begin + 63) >> 6;
+        float* st_out = p.out_state ? p.out_state + ((size_t)n * p.Hv + h) * 128 * 128 : nullptr;
+        if (nchunks == 0) {                                   // empty request: zero state, no outputs
+            if (st_out) for (int a = 0; a < 64; ++a) st_out[(64 * hf + a) * 128 + dv] = 0.f;
+            continue;
+        }
+#pragma unroll 1
+        for (int c = 0; c < nchunks; ++c, ++j) {
+            const int row0 = row_begin + c * 64;
+            const int nvalid = min(64, row_end - row0);
+            const bool first = c == 0, last = c == nchunks - 1;
+            const Decay& dc = misc->decay[j & 3u];
+            GDN_DBG(const bool dbg = prm.debug && blockIdx.x == 0 && r == 0 && c < 2; float* dbase = prm.debug + c * DBG_STRIDE;)
+
+            // total log-decay of the next chunk (scales the carried state ahead of its update MMA)
+            float eGCnext = 1.f;
+            if (!last) {
+                const int nrow0 = row0 + 64, nnv = min(64, row_end - nrow0);
+                float gs = (lane < nnv ? p.g[(size_t)(nrow0 + lane) * p.Hv + h] : 0.f) +
+                           (lane + 32 < nnv ? p.g[(size_t)(nrow0 + lane + 32) * p.Hv + h] : 0.f);
+#pragma unroll
+                for (int off = 16; off > 0; off >>= 1) gs += __shfl_xor_sync(0xffffffffu, gs, off);
+                eGCnext = ex2_approx(gs * kLog2e);
+            }
+
+            // ---- Delta epilogue: bf16 Delta^T and decayed Delta'^T as TMEM A operands ----------------------
+            cx.wait(B_PRE_DONE0 + (j & 1u), (j >> 1) & 1u);      // decay factors of this chunk are published
+            GDN_T(0);
+            cx.wait(B_MMA1_DONE, j & 1u);
+            GDN_T(1);
+            tc_fence_after();
+#pragma unroll 1
+            for (int g = 0; g < 2; ++g) {
+                const int c0 = 32 * hf + 16 * g;
+                uint32_t acc[16], d1[8], d2[8];
+                tmem_ld16(tl + TM_ACC1 + c0, acc);
+                tmem_ld_wait();
+#ifdef GDN_TC_DEBUG
+                if (dbg) {
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) dbase[20480 + dv * 64 + c0 + i] = __uint_as_float(acc[i]);
+                }
+#endif
+#pragma unroll
+                for (int i4 = 0; i4 < 4; ++i4) {
+                    const float4 er = *reinterpret_cast<const float4*>(&dc.eRest[c0 + 4 * i4]);
+                    const float a0 = __uint_as_float(acc[4 * i4]), a1 = __uint_as_float(acc[4 * i4 + 1]);
+                    const float a2 = __uint_as_float(acc[4 * i4 + 2]), a3 = __uint_as_float(acc[4 * i4 + 3]);
+                    d1[2 * i4] = pack_bf16x2(a0, a1);
+                    d1[2 * i4 + 1] = pack_bf16x2(a2, a3);
+                    d2[2 * i4] = pack_bf16x2(a0 * er.x, a1 * er.y);
+                    d2[2 * i4 + 1] = pack_bf16x2(a2 * er.z, a3 * er.w);
+                }
+                tmem_st8(tl + TM_DBF + (c0 >> 1), d1);
+                tmem_st8(tl + TM_DPBF + (c0 >> 1), d2);
+            }
+            tmem_st_wait();
+            tc_fence_before();
+            mbar_arrive(cx.bar(B_D_READY));
+            GDN_T(2);
+
+            // ---- state: bf16 copy for the next chunk's MMAs + pre-scaling, or the final state ----------------
+            cx.wait(B_MMA3_DONE, j & 1u);
+            GDN_T(3);
+            tc_fence_after();
+#pragma unroll 1
+            for (int g = 0; g < 4; ++g) {
+                const int c0 = 64 * hf + 16 * g;
+                uint32_t acc[16];
+                tmem_ld16(tl + TM_S32 + c0, acc);
+                tmem_ld_wait();
+#ifdef GDN_TC_DEBUG
+                if (dbg) {
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) dbase[45056 + dv * 128 + c0 + i] = __uint_as_float(acc[i]);
+                }
+#endif
+                if (!last) {
+                    uint32_t pk[8];
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) pk[i] = pack_bf16x2(__uint_as_float(acc[2 * i]), __uint_as_float(acc[2 * i + 1]));
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) acc[i] = __float_as_uint(__uint_as_float(acc[i]) * eGCnext);
+                    tmem_st8(tl + TM_SBF + (c0 >> 1), pk);
+                    tmem_st16(tl + TM_S32 + c0, acc);
+                } else if (st_out) {
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) st_out[(c0 + i) * 128 + dv] = __uint_as_float(acc[i]);
+                }
+            }
+            tmem_st_wait();
+            tc_fence_before();
+            mbar_arrive(cx.bar(B_SBF_READY));
+            GDN_T(4);
+
+            // ---- output epilogue: O^T = diag(e^G) (S0 Q^T) + Delta^T P^T, transposed through shared memory ----
+            {
+                __nv_bfloat16* ost = reinterpret_cast<__nv_bfloat16*>(cx.sm + SM_OST);
+                if (og) wg_sync(2);                            // previous chunk's staged tile fully drained
+                GDN_T(5);
+#pragma unroll 1
+                for (int g = 0; g < 2; ++g) {
+                    const int c0 = 32 * hf + 16 * g;
+                    uint32_t a3[16], a2[16];
+                    tmem_ld16(tl + TM_ACC3 + c0, a3);
+                    if (!first) tmem_ld16(tl + TM_ACC2 + c0, a2);
+                    tmem_ld_wait();
+#ifdef GDN_TC_DEBUG
+                    if (dbg) {
+#pragma unroll
+                        for (int i = 0; i < 16; ++i) {
+                            dbase[36864 + dv * 64 + c0 + i] = __uint_as_float(a3[i]);
+                            dbase[28672 + dv * 64 + c0 + i] = !first ? __uint_as_float(a2[i]) : 0.f;
+                        }
+                    }
+#endif
+                    if (og) {
+#pragma unroll
+                        for (int i4 = 0; i4 < 4; ++i4) {
+                            const float4 eg = *reinterpret_cast<const float4*>(&dc.eG[c0 + 4 * i4]);
+                            const float egs[4] = {eg.x, eg.y, eg.z, eg.w};
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) {
+                                const int i = 4 * i4 + e;
+                                float o = __uint_as_float(a3[i]);
+                                if (!first) o = fmaf(egs[e], __uint_as_float(a2[i]), o);
+                                ost[(c0 + i) * 128 + dv] = __float2bfloat16_rn(o);
+                            }
+                        }
+                    }
+                }
+                tc_fence_before();
+                mbar_arrive(cx.bar(B_ACC23_FREE));
+                GDN_T(6);
+                if (og) {
+                    wg_sync(2);
+                    GDN_T(7);
+                    const uint4* src = reinterpret_cast<const uint4*>(cx.sm + SM_OST);
+#pragma unroll
+                    for (int it = 0; it < 4; ++it) {
+                        const int idx = it * kWgThreads + wtid, row = idx >> 4, c16 = idx & 15;
+                        if (row < nvalid)
+                            *reinterpret_cast<uint4*>(reinterpret_cast<uint8_t*>(og) + (((size_t)(row0 + row) * p.Hv + h) * 256 + c16 * 16)) = src[idx];
+                    }
+                }
+            }
+            GDN_T(8);
+            GDN_DBG(++nch;)
+        }
+    }
+#ifdef GDN_TC_DEBUG
+    if (prm.debug && blockIdx.x == 0 && wtid == 0 && nch > 0) {
+        float* d = prm.debug + 2 * DBG_STRIDE + 16;
+        d[0] = (float)nch;
+        for (int i = 0; i < 12; ++i) d[1 + i] = (float)tt_[i] / nch;
+    }
+#endif
+}
+
+__global__ void __launch_bounds__(kThreads, 1)
 gdn_tc_kernel(const TcParams prm, const __grid_constant__ CUtensorMap tm_q,
               const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v)
 {
     extern __shared__ uint8_t smem_raw[];
-    const Problem& p = prm.p;
     const uint32_t raw = smem_u32(smem_raw);
-    const uint32_t sb = (raw + 1023u) & ~1023u;           // shared-space address of the aligned base
-    uint8_t* sm = smem_raw + (sb - raw);                  // generic pointer to the same place
-    Misc* misc = reinterpret_cast<Misc*>(sm + SM_MISC);
-    float* AF = reinterpret_cast<float*>(sm + SM_AF);
-    float* XF = reinterpret_cast<float*>(sm + SM_XF);
-    float* MF = reinterpret_cast<float*>(sm + SM_MF);
+    Ctx cx;
+    cx.sb = (raw + 1023u) & ~1023u;
+    cx.sm = smem_raw + (cx.sb - raw);
+    cx.misc = reinterpret_cast<Misc*>(cx.sm + SM_MISC);
 
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const uint32_t bar_tma = sb + SM_MISC + offsetof(Misc, bar_tma);
-    const uint32_t bar_mma = sb + SM_MISC + offsetof(Misc, bar_mma);
-
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     if (warp == 0) {
-        tmem_alloc(sb + SM_MISC + offsetof(Misc, tmem_base), 512);
+        tmem_alloc(cx.sb + SM_MISC + (uint32_t)offsetof(Misc, tmem_base), 512);
         tmem_relinquish();
     }
-    if (tid == 0) {
-        mbar_init(bar_tma, 1);
-        mbar_init(bar_mma, 1);
+    if (tid == 32) {
+        for (int i = 0; i < NUM_BARS; ++i) {
+            const bool wg_bar = i == B_WACC_READ || i == B_TPP_READY || i == B_PRE_DONE0 || i == B_PRE_DONE1 ||
+                                i == B_D_READY || i == B_SBF_READY || i == B_ACC23_FREE;
+            mbar_init(cx.bar(i), wg_bar ? (uint32_t)kWgThreads : 1u);
+        }
         fence_mbar_init();
-        misc->abort = 0;
+        cx.misc->abort = 0u;
         prefetch_tmap(&tm_q); prefetch_tmap(&tm_k); prefetch_tmap(&tm_v);
     }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
-    const uint32_t tmem = misc->tmem_base;
-    const uint32_t tl = tmem + ((uint32_t)(warp * 32) << 16);     // this warp's lane window
-    uint32_t ph_tma = 0, ph_mma = 0;
-    bool aborted = false;
+    cx.tmem = cx.misc->tmem_base;
 
-    const int G = p.Hv / p.Hq;
-    const uint32_t num_items = (uint32_t)p.num_seqs * (uint32_t)p.Hv;
-    __nv_bfloat16* __restrict__ og = reinterpret_cast<__nv_bfloat16*>(p.out_o);
-
-    // Waits (bounded) on an mbarrier with all threads, then agrees on success across the CTA.
-    auto wait_all = [&](uint32_t bar, uint32_t& phase) -> bool {
-        if (!mbar_wait_bounded(bar, phase)) misc->abort = 1;
-        phase ^= 1u;
-        __syncthreads();
-        return misc->abort == 0;
-    };
-
-    for (;;) {
-        if (tid == 0) misc->item = atomicAdd(&prm.s.header->next_item, 1u);
-        __syncthreads();
-        const uint32_t item = misc->item;
-        if (item >= num_items) break;
-        const int n = prm.s.order[item / p.Hv];
-        const int h = item % p.Hv;
-        const int hq = h / G;
-        const int row_begin = p.cu[n], row_end = p.cu[n + 1];
-        const int nchunks = (row_end - row_begin + 63) >> 6;
-        float* st_out = p.out_state ? p.out_state + ((size_t)n * p.Hv + h) * 128 * 128 : nullptr;
-
-        for (int c = 0; c < nchunks; ++c) {
-            const int row0 = row_begin + c * 64;
-            const int nvalid = min(64, row_end - row0);
-
-            // ---- A. TMA loads of the K, Q, V tiles of this chunk --------------------------------
-            if (tid == 0) {
-                mbar_arrive_expect_tx(bar_tma, 49152u);
-                tma_load_2d(sb + SM_KQ, &tm_k, hq * 128, row0, bar_tma);
-                tma_load_2d(sb + SM_KQ + 16384, &tm_k, hq * 128 + 64, row0, bar_tma);
-                tma_load_2d(sb + SM_KQ + 8192, &tm_q, hq * 128, row0, bar_tma);
-                tma_load_2d(sb + SM_KQ + 24576, &tm_q, hq * 128 + 64, row0, bar_tma);
-                tma_load_2d(sb + SM_V, &tm_v, h * 128, row0, bar_tma);
-                tma_load_2d(sb + SM_V + 8192, &tm_v, h * 128 + 64, row0, bar_tma);
-            }
-            // ---- B. log-decay cumsum and the decay factors ---------------------------------------
-            if (tid < 64) {
-                const bool ok = tid < nvalid;
-                misc->g[tid] = ok ? p.g[(size_t)(row0 + tid) * p.Hv + h] : 0.f;
-                misc->beta[tid] = ok ? p.beta[(size_t)(row0 + tid) * p.Hv + h] : 0.f;
-            }
-            __syncthreads();
-            if (tid < 64) {
-                float acc = 0.f;
-                for (int s2 = 0; s2 <= tid; ++s2) acc += misc->g[s2];
-                misc->G[tid] = acc;
-            }
-            __syncthreads();
-            const float GC = misc->G[63];
-            if (tid < 64) {
-                const float Gt = misc->G[tid];
-                misc->eG[tid] = ex2_approx(Gt * kLog2e);
-                misc->eRest[tid] = ex2_approx((GC - Gt) * kLog2e);
-            }
-            const float eGC = ex2_approx(GC * kLog2e);
-
-            // ---- C. chunk-start state: bf16 copy for the MMAs, fp32 master pre-scaled by e^{G_C} ----
-            if (c > 0) {
-                tc_fence_after();
-#pragma unroll
-                for (int hf = 0; hf < 2; ++hf) {
-                    uint32_t r0[32], r1[32], pk[32];
-                    tmem_ld32(tl + TM_S32 + hf * 64, r0);
-                    tmem_ld32(tl + TM_S32 + hf * 64 + 32, r1);
-                    tmem_ld_wait();
-#pragma unroll
-                    for (int i = 0; i < 16; ++i) {
-                        pk[i] = pack_bf16x2(__uint_as_float(r0[2 * i]), __uint_as_float(r0[2 * i + 1]));
-                        pk[16 + i] = pack_bf16x2(__uint_as_float(r1[2 * i]), __uint_as_float(r1[2 * i + 1]));
-                    }
-#pragma unroll
-                    for (int i = 0; i < 32; ++i) {
-                        r0[i] = __float_as_uint(__uint_as_float(r0[i]) * eGC);
-                        r1[i] = __float_as_uint(__uint_as_float(r1[i]) * eGC);
-                    }
-                    tmem_st32(tl + TM_SBF + hf * 32, pk);
-                    tmem_st32(tl + TM_S32 + hf * 64, r0);
-                    tmem_st32(tl + TM_S32 + hf * 64 + 32, r1);
-                }
-                tmem_st_wait();
-                tc_fence_before();
-            }
-
-            // ---- D. Gram MMA: [K;Q] K^T -> TM_GRAM ----------------------------------------------------
-            if (!wait_all(bar_tma, ph_tma)) { aborted = true; break; }
-            if (tid == 0) {
-                tc_fence_after();
-#pragma unroll
-                for (int ks = 0; ks < 8; ++ks) {
-                    const uint32_t a = sb + SM_KQ + (ks >> 2) * 16384 + (ks & 3) * 32;
-                    mma_ss(tmem + TM_GRAM, smem_desc_sw128(a, 16, 1024), smem_desc_sw128(a, 16, 1024), ID_GRAM, ks > 0);
-                }
-                mma_commit(bar_mma);
-            }
-            if (!wait_all(bar_mma, ph_mma)) { aborted = true; break; }
-            tc_fence_after();
-
-            // ---- E. A (fp32, shared) and P (bf16 operand) from the Gram tile ---------------------------
-            {
-                uint32_t r0[32], r1[32];
-                tmem_ld32(tl + TM_GRAM, r0);
-                tmem_ld32(tl + TM_GRAM + 32, r1);
-                tmem_ld_wait();
-                const int t = tid & 63;
-                const float Gt = misc->G[t];
-                if (tid < 64) {
-                    const float bt = misc->beta[t];
-#pragma unroll
-                    for (int s2 = 0; s2 < 64; ++s2) {
-                        const float acc = __uint_as_float(s2 < 32 ? r0[s2 & 31] : r1[s2 & 31]);
-                        const float arg = (s2 < t) ? (Gt - misc->G[s2]) * kLog2e : 0.f;
-                        AF[t * LDF + s2] = (s2 < t) ? bt * ex2_approx(arg) * acc : 0.f;
-                    }
-                } else {
-                    uint8_t* prow = sm + SM_P + t * 128;
-#pragma unroll
-                    for (int ch = 0; ch < 8; ++ch) {
-                        uint32_t w[4];
-#pragma unroll
-                        for (int e = 0; e < 4; ++e) {
-                            float v2[2];
-#pragma unroll
-                            for (int u = 0; u < 2; ++u) {
-                                const int s2 = ch * 8 + e * 2 + u;
-                                const float acc = __uint_as_float(s2 < 32 ? r0[s2 & 31] : r1[s2 & 31]);
-                                const float arg = (s2 <= t) ? (Gt - misc->G[s2]) * kLog2e : 0.f;
-                                v2[u] = (s2 <= t) ? ex2_approx(arg) * acc : 0.f;
-                            }
-                            w[e] = pack_bf16x2(v2[0], v2[1]);
-                        }
-                        *reinterpret_cast<uint4*>(prow + ((ch ^ (t & 7)) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
-                    }
-                }
-            }
-#ifdef GDN_TC_DEBUG
-            if (prm.debug && item == 0 && c < 2) {
-                uint32_t r0[32], r1[32];
-                tmem_ld32(tl + TM_GRAM, r0); tmem_ld32(tl + TM_GRAM + 32, r1); tmem_ld_wait();
-                float* d = prm.debug + c * DBG_STRIDE;
-                for (int i = 0; i < 32; ++i) { d[tid * 64 + i] = __uint_as_float(r0[i]); d[tid * 64 + 32 + i] = __uint_as_float(r1[i]); }
-            }
-#endif
-            tc_fence_before();
-            __syncthreads();
-
-            // ---- F. X = (I + A)^-1: 16 x 16 diagonal blocks by substitution, then block rows ----------
-            if (lane < 16) {
-                const int b = warp * 16, j = lane;
-                float x[16];
-#pragma unroll
-                for (int r = 0; r < 16; ++r) x[r] = (r == j) ? 1.f : 0.f;
-#pragma unroll
-                for (int r = 1; r < 16; ++r) {
-                    float acc = 0.f;
-#pragma unroll
-                    for (int s2 = 0; s2 < r; ++s2) acc = fmaf(AF[(b + r) * LDF + b + s2], x[s2], acc);
-                    x[r] = (r > j) ? -acc : x[r];
-                }
-#pragma unroll
-                for (int r = 0; r < 16; ++r) XF[(b + r) * LDF + b + j] = x[r];
-            }
-            __syncthreads();
-            for (int I = 1; I < 4; ++I) {
-                const int ncol = 16 * I;
-                for (int e = tid; e < 16 * ncol; e += 128) {
-                    const int r = e / ncol, cc = e % ncol;
-                    float acc = 0.f;
-                    for (int m = cc & ~15; m < ncol; ++m) acc = fmaf(AF[(ncol + r) * LDF + m], XF[m * LDF + cc], acc);
-                    MF[r * 64 + cc] = acc;
-                }
-                __syncthreads();
-                for (int e = tid; e < 16 * ncol; e += 128) {
-                    const int r = e / ncol, cc = e % ncol;
-                    float acc = 0.f;
-#pragma unroll
-                    for (int m = 0; m < 16; ++m) acc = fmaf(XF[(ncol + r) * LDF + ncol + m], MF[m * 64 + cc], acc);
-                    XF[(ncol + r) * LDF + cc] = -acc;
-                }
-                __syncthreads();
-            }
-            // T' = X diag(beta), T'' = X diag(beta e^G) as bf16 K-major operands
-            {
-                const int t = tid >> 1, hf = tid & 1;
-#pragma unroll
-                for (int ch = 0; ch < 4; ++ch) {
-                    uint32_t w1[4], w2[4];
-#pragma unroll
-                    for (int e = 0; e < 4; ++e) {
-                        float a1[2], a2[2];
-#pragma unroll
-                        for (int u = 0; u < 2; ++u) {
-                            const int s2 = hf * 32 + ch * 8 + e * 2 + u;
-                            const float x = (s2 <= t) ? XF[t * LDF + s2] : 0.f;
-                            a1[u] = x * misc->beta[s2];
-                            a2[u] = a1[u] * misc->eG[s2];
-                        }
-                        w1[e] = pack_bf16x2(a1[0], a1[1]);
-                        w2[e] = pack_bf16x2(a2[0], a2[1]);
-                    }
-                    const int chunk16 = hf * 4 + ch;
-                    const uint32_t off = t * 128 + ((chunk16 ^ (t & 7)) << 4);
-                    *reinterpret_cast<uint4*>(sm + SM_TP + off) = make_uint4(w1[0], w1[1], w1[2], w1[3]);
-                    *reinterpret_cast<uint4*>(sm + SM_TPP + off) = make_uint4(w2[0], w2[1], w2[2], w2[3]);
-                }
-            }
-#ifdef GDN_TC_DEBUG
-            if (prm.debug && item == 0 && c < 2) {
-                float* d = prm.debug + c * DBG_STRIDE + 8192;
-                for (int e = tid; e < 4096; e += 128) d[e] = ((e & 63) <= (e >> 6)) ? XF[(e >> 6) * LDF + (e & 63)] : 0.f;
-            }
-#endif
-            fence_proxy_async_smem();
-            __syncthreads();
-
-            // ---- G. W^T = K^T T''^T -> TM_GRAM,  U^T = V^T T'^T -> TM_ACC1 -----------------------------
-            if (tid == 0) {
-                tc_fence_after();
-#pragma unroll
-                for (int ks = 0; ks < 4; ++ks) {
-                    mma_ss(tmem + TM_GRAM, smem_desc_sw128(sb + SM_KQ + ks * 2048, 16384, 1024),
-                           smem_desc_sw128(sb + SM_TPP + ks * 32, 16, 1024), ID_WU, ks > 0);
-                }
-#pragma unroll
-                for (int ks = 0; ks < 4; ++ks) {
-                    mma_ss(tmem + TM_ACC1, smem_desc_sw128(sb + SM_V + ks * 2048, 8192, 1024),
-                           smem_desc_sw128(sb + SM_TP + ks * 32, 16, 1024), ID_WU, ks > 0);
-                }
-                mma_commit(bar_mma);
-            }
-            if (!wait_all(bar_mma, ph_mma)) { aborted = true; break; }
-            tc_fence_after();
-
-            // ---- H. W epilogue: W[t][dk] bf16 into shared memory as a K-major operand ------------------
-            {
-                uint32_t r0[32], r1[32];
-                tmem_ld32(tl + TM_GRAM, r0);
-                tmem_ld32(tl + TM_GRAM + 32, r1);
-                tmem_ld_wait();
-#ifdef GDN_TC_DEBUG
-                if (prm.debug && item == 0 && c < 2) {
-                    float* d = prm.debug + c * DBG_STRIDE + 12288;
-                    for (int i = 0; i < 32; ++i) { d[tid * 64 + i] = __uint_as_float(r0[i]); d[tid * 64 + 32 + i] = __uint_as_float(r1[i]); }
-                }
-#endif
-                const int dd = tid & 63;
-                uint8_t* wbase = sm + SM_W + (tid >> 6) * 8192 + (dd & 7) * 2;
-#pragma unroll
-                for (int t = 0; t < 64; ++t) {
-                    const float wv = __uint_as_float(t < 32 ? r0[t & 31] : r1[t & 31]);
-                    *reinterpret_cast<__nv_bfloat16*>(wbase + t * 128 + (((dd >> 3) ^ (t & 7)) << 4)) = __float2bfloat16_rn(wv);
-                }
-            }
-            fence_proxy_async_smem();
-            tc_fence_before();
-            __syncthreads();
-
-            // ---- I. Delta^T = U^T - S0 W^T (onto TM_ACC1),  S0 Q^T -> TM_ACC2 -------------------------
-            if (c > 0) {
-                if (tid == 0) {
-                    tc_fence_after();
-#pragma unroll
-                    for (int ks = 0; ks < 8; ++ks) {
-                        mma_ts(tmem + TM_ACC1, tmem + TM_SBF + ks * 8,
-                               smem_desc_sw128(sb + SM_W + (ks >> 2) * 8192 + (ks & 3) * 32, 16, 1024), ID_SW, 1u);
-                    }
-#pragma unroll
-                    for (int ks = 0; ks < 8; ++ks) {
-                        mma_ts(tmem + TM_ACC2, tmem + TM_SBF + ks * 8,
-                               smem_desc_sw128(sb + SM_KQ + 8192 + (ks >> 2) * 16384 + (ks & 3) * 32, 16, 1024), ID_SQ, ks > 0);
-                    }
-                    mma_commit(bar_mma);
-                }
-                if (!wait_all(bar_mma, ph_mma)) { aborted = true; break; }
-                tc_fence_after();
-            }
-
-            // ---- J. Delta epilogue: bf16 Delta^T and decayed Delta'^T as TMEM A operands ----------------
-            {
-                uint32_t r0[32], r1[32], d1[32], d2[32];
-                tmem_ld32(tl + TM_ACC1, r0);
-                tmem_ld32(tl + TM_ACC1 + 32, r1);
-                tmem_ld_wait();
-#ifdef GDN_TC_DEBUG
-                if (prm.debug && item == 0 && c < 2) {
-                    float* d = prm.debug + c * DBG_STRIDE + 20480;
-                    for (int i = 0; i < 32; ++i) { d[tid * 64 + i] = __uint_as_float(r0[i]); d[tid * 64 + 32 + i] = __uint_as_float(r1[i]); }
-                }
-#endif
-#pragma unroll
-                for (int i = 0; i < 16; ++i) {
-                    const float a0 = __uint_as_float(r0[2 * i]), a1 = __uint_as_float(r0[2 * i + 1]);
-                    const float b0 = __uint_as_float(r1[2 * i]), b1 = __uint_as_float(r1[2 * i + 1]);
-                    d1[i] = pack_bf16x2(a0, a1);
-                    d1[16 + i] = pack_bf16x2(b0, b1);
-                    d2[i] = pack_bf16x2(a0 * misc->eRest[2 * i], a1 * misc->eRest[2 * i + 1]);
-                    d2[16 + i] = pack_bf16x2(b0 * misc->eRest[32 + 2 * i], b1 * misc->eRest[32 + 2 * i + 1]);
-                }
-                tmem_st32(tl + TM_DBF, d1);
-                tmem_st32(tl + TM_DPBF, d2);
-                tmem_st_wait();
-            }
-            tc_fence_before();
-            __syncthreads();
-
-            // ---- K. Delta^T P^T -> TM_ACC3,  S += Delta'^T K (onto the pre-scaled TM_S32) --------------
-            if (tid == 0) {
-                tc_fence_after();
-#pragma unroll
-                for (int ks = 0; ks < 4; ++ks) {
-                    mma_ts(tmem + TM_ACC3, tmem + TM_DBF + ks * 8,
-                           smem_desc_sw128(sb + SM_P + ks * 32, 16, 1024), ID_DP, ks > 0);
-                }
-#pragma unroll
-                for (int ks = 0; ks < 4; ++ks) {
-                    mma_ts(tmem + TM_S32, tmem + TM_DPBF + ks * 8,
-                           smem_desc_sw128(sb + SM_KQ + ks * 2048, 16384, 1024), ID_DK, (c > 0 || ks > 0) ? 1u : 0u);
-                }
-                mma_commit(bar_mma);
-            }
-            if (!wait_all(bar_mma, ph_mma)) { aborted = true; break; }
-            tc_fence_after();
-
-            // ---- L. output epilogue: O^T = diag(e^G) (S0 Q^T) + Delta^T P^T, stored for valid rows -----
-            if (og) {
-                uint32_t r0[32], r1[32], q0[32], q1[32];
-                tmem_ld32(tl + TM_ACC3, r0);
-                tmem_ld32(tl + TM_ACC3 + 32, r1);
-                if (c > 0) {
-                    tmem_ld32(tl + TM_ACC2, q0);
-                    tmem_ld32(tl + TM_ACC2 + 32, q1);
-                }
-                tmem_ld_wait();
-#ifdef GDN_TC_DEBUG
-                if (prm.debug && item == 0 && c < 2) {
-                    float* d = prm.debug + c * DBG_STRIDE;
-                    for (int i = 0; i < 32; ++i) {
-                        d[36864 + tid * 64 + i] = __uint_as_float(r0[i]); d[36864 + tid * 64 + 32 + i] = __uint_as_float(r1[i]);
-                        d[28672 + tid * 64 + i] = c > 0 ? __uint_as_float(q0[i]) : 0.f;
-                        d[28672 + tid * 64 + 32 + i] = c > 0 ? __uint_as_float(q1[i]) : 0.f;
-                    }
-                }
-#endif
-                __nv_bfloat16* orow = og + ((size_t)row0 * p.Hv + h) * 128 + tid;
-#pragma unroll
-                for (int t = 0; t < 64; ++t) {
-                    float o = __uint_as_float(t < 32 ? r0[t & 31] : r1[t & 31]);
-                    if (c > 0) o = fmaf(misc->eG[t], __uint_as_float(t < 32 ? q0[t & 31] : q1[t & 31]), o);
-                    if (t < nvalid) orow[(size_t)t * p.Hv * 128] = __float2bfloat16_rn(o);
-                }
-            }
-#ifdef GDN_TC_DEBUG
-            if (prm.debug && item == 0 && c < 2) {
-                float* d = prm.debug + c * DBG_STRIDE + 45056;
-                for (int q4 = 0; q4 < 4; ++q4) {
-                    uint32_t r0[32];
-                    tmem_ld32(tl + TM_S32 + q4 * 32, r0); tmem_ld_wait();
-                    for (int i = 0; i < 32; ++i) d[tid * 128 + q4 * 32 + i] = __uint_as_float(r0[i]);
-                }
-            }
-#endif
-            tc_fence_before();
-            __syncthreads();
-        }
-        if (aborted) break;
-
-        // ---- final state: out_state[n, h, a, b] = S[b][a] --------------------------------------------
-        if (st_out) {
-            if (nchunks == 0) {
-                for (int a = 0; a < 128; ++a) st_out[a * 128 + tid] = 0.f;
-            } else {
-                tc_fence_after();
-#pragma unroll
-                for (int q4 = 0; q4 < 4; ++q4) {
-                    uint32_t r0[32];
-                    tmem_ld32(tl + TM_S32 + q4 * 32, r0);
-                    tmem_ld_wait();
-#pragma unroll
-                    for (int i = 0; i < 32; ++i) st_out[(q4 * 32 + i) * 128 + tid] = __uint_as_float(r0[i]);
-                }
-                tc_fence_before();
-            }
-        }
-        __syncthreads();
+    if (warp == 0) {
+        if (lane == 0) role_producer(cx, prm, &tm_q, &tm_k, &tm_v);
+    } else if (warp == 1) {
+        if (lane == 0) role_mma_chain(cx, prm);
+    } else if (warp == 2) {
+        if (lane == 0) role_mma_pre(cx, prm);
+    } else if (warp >= 4 && warp < 12) {
+        role_pre(cx, prm, tid - 128);
+    } else if (warp >= 12) {
+        role_chain(cx, prm, tid - 384);
     }
 
-    if (aborted) {
-        if (tid == 0 && p.status_word) *p.status_word = GDN_ERR_TIMEOUT;
-        // give copies that may still be in flight a bounded chance to land before the CTA retires
-        if (tid == 0) mbar_wait_bounded(bar_tma, ph_tma ^ 1u, 200000000ull);
-    }
     tc_fence_before();
     __syncthreads();
-    if (warp == 0) tmem_dealloc(tmem, 512);
+    if (cx.misc->abort) {
+        // let copies and MMAs that may still be in flight land before shared and tensor memory are released
+        for (int i = 0; i < 1000; ++i) __nanosleep(1000);
+        if (tid == 0 && prm.p.status_word) *prm.p.status_word = GDN_ERR_TIMEOUT;
+        __syncthreads();
+    }
+    if (warp == 0) tmem_dealloc(cx.tmem, 512);
 }
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
@@ -577,7 +902,7 @@ cudaError_t launch_tcgen05(const Problem& p, const Sched& s, cudaStream_t stream
     if (grid > sms) grid = sms;
     TcParams prm;
     prm.p = p; prm.s = s; prm.debug = g_debug_buffer;
-    gdn_tc_kernel<<<(unsigned)grid, 128, SMEM_BYTES, stream>>>(prm, tq, tk, tv);
+    gdn_tc_kernel<<<(unsigned)grid, kThreads, SMEM_BYTES, stream>>>(prm, tq, tk, tv);
     e = cudaGetLastError();
     if (e == cudaSuccess && launches) *launches += 1;
     return e;
