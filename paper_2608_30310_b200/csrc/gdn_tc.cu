@@ -165,7 +165,26 @@ struct Ctx {
     // Bounded wait.  On expiry it raises the CTA-wide abort flag; from then on no wait blocks any more, so
     // every role still runs through its (data-independent) loop structure, keeps meeting its warpgroup
     // barriers and reaches the end of the kernel; the results are garbage and the host sees the status word.
+#ifdef GDN_TC_PROFILE
+    mutable long long wait_cycles[NUM_BARS];
+    mutable long long t_begin;
+    __device__ void prof_init() const { for (int i = 0; i < NUM_BARS; ++i) wait_cycles[i] = 0; t_begin = clock64(); }
+    __device__ void prof_dump(float* dst) const
+    {
+        dst[0] = (float)(clock64() - t_begin);
+        for (int i = 0; i < NUM_BARS; ++i) dst[1 + i] = (float)wait_cycles[i];
+    }
     __device__ bool wait(int i, uint32_t parity) const
+    {
+        const long long c0 = clock64();
+        const bool r = wait_impl(i, parity);
+        wait_cycles[i] += clock64() - c0;
+        return r;
+    }
+    __device__ bool wait_impl(int i, uint32_t parity) const
+#else
+    __device__ bool wait(int i, uint32_t parity) const
+#endif
     {
         const uint32_t b = bar(i);
         if (mbar_try_wait(b, parity)) return true;
@@ -183,6 +202,13 @@ struct Ctx {
 };
 
 __device__ __forceinline__ void wg_sync(int id) { asm volatile("bar.sync %0, 256;" ::"r"(id) : "memory"); }
+// One arrival per warp: every lane has fenced its own TMEM / shared-memory accesses, the warp converges,
+// lane 0 arrives.  (A full-warp arrive is 32 serialized shared-memory atomics on one address.)
+__device__ __forceinline__ void warp_arrive(uint32_t bar, int lane)
+{
+    __syncwarp();
+    if (lane == 0) mbar_arrive(bar);
+}
 __device__ __forceinline__ uint32_t to_tf32(float x)
 {
     uint32_t r;
@@ -232,11 +258,14 @@ __device__ void role_producer(const Ctx& cx, const TcParams& prm, const CUtensor
     cv = ckq;
     auto load_kq = [&](const ChunkCursor& cc, uint32_t j) {
         const uint32_t slot = j % 3u, dst = cx.sb + SM_KQ + slot * KQ_SLOT, bar = cx.bar(B_FULL_KQ0 + slot);
-        mbar_arrive_expect_tx(bar, 32768u);
-        tma_load_2d(dst, tm_k, cc.hq * 128, cc.row0(), bar);
-        tma_load_2d(dst + 16384, tm_k, cc.hq * 128 + 64, cc.row0(), bar);
-        tma_load_2d(dst + 8192, tm_q, cc.hq * 128, cc.row0(), bar);
-        tma_load_2d(dst + 24576, tm_q, cc.hq * 128 + 64, cc.row0(), bar);
+        if (elect_one()) {
+            mbar_arrive_expect_tx(bar, 32768u);
+            tma_load_2d(dst, tm_k, cc.hq * 128, cc.row0(), bar);
+            tma_load_2d(dst + 16384, tm_k, cc.hq * 128 + 64, cc.row0(), bar);
+            tma_load_2d(dst + 8192, tm_q, cc.hq * 128, cc.row0(), bar);
+            tma_load_2d(dst + 24576, tm_q, cc.hq * 128 + 64, cc.row0(), bar);
+        }
+        __syncwarp();
     };
     uint32_t jkq = 0;
     for (; jkq < 2 && ckq.valid; ++jkq) { load_kq(ckq, jkq); ckq.advance(); }
@@ -245,9 +274,12 @@ __device__ void role_producer(const Ctx& cx, const TcParams& prm, const CUtensor
         // V(j): the single slot is free once U^T MMA of chunk j-1 has completed
         if (j >= 1) cx.wait(B_U_DONE, (j - 1) & 1u);
         const uint32_t bar = cx.bar(B_FULL_V);
-        mbar_arrive_expect_tx(bar, 16384u);
-        tma_load_2d(cx.sb + SM_V, tm_v, cv.h * 128, cv.row0(), bar);
-        tma_load_2d(cx.sb + SM_V + 8192, tm_v, cv.h * 128 + 64, cv.row0(), bar);
+        if (elect_one()) {
+            mbar_arrive_expect_tx(bar, 16384u);
+            tma_load_2d(cx.sb + SM_V, tm_v, cv.h * 128, cv.row0(), bar);
+            tma_load_2d(cx.sb + SM_V + 8192, tm_v, cv.h * 128 + 64, cv.row0(), bar);
+        }
+        __syncwarp();
         cv.advance();
         // K/Q(j+2): its slot held chunk j-1, free once the state-update MMA of chunk j-1 has completed
         if (ckq.valid) {
@@ -278,18 +310,24 @@ __device__ void role_mma_pre(const Ctx& cx, const TcParams& prm)
         cx.wait(B_FULL_KQ0 + slot, (j / 3u) & 1u);
         if (j >= 1) cx.wait(B_WACC_READ, (j - 1) & 1u);
         tc_fence_after();
-#pragma unroll 1
-        for (int ks = 0; ks < 8; ++ks) {
-            const uint64_t d = desc_add(d_kq, (ks >> 2) * 16384 + (ks & 3) * 32);
-            mma_ss(cx.tmem + TM_GRAM, d, d, ID_GRAM, ks > 0);
+        if (elect_one()) {
+#pragma unroll
+            for (int ks = 0; ks < 8; ++ks) {
+                const uint64_t d = desc_add(d_kq, (ks >> 2) * 16384 + (ks & 3) * 32);
+                mma_ss(cx.tmem + TM_GRAM, d, d, ID_GRAM, ks > 0);
+            }
+            mma_commit(cx.bar(B_GRAM_DONE));
         }
-        mma_commit(cx.bar(B_GRAM_DONE));
+        __syncwarp();
         cx.wait(B_TPP_READY, j & 1u);
         tc_fence_after();
-#pragma unroll 1
-        for (int ks = 0; ks < 4; ++ks)
-            mma_ss(cx.tmem + TM_GRAM, desc_add(d_kt, ks * 2048), desc_add(d_tpp, ks * 32), ID_WU, ks > 0);
-        mma_commit(cx.bar(B_W_DONE));
+        if (elect_one()) {
+#pragma unroll
+            for (int ks = 0; ks < 4; ++ks)
+                mma_ss(cx.tmem + TM_GRAM, desc_add(d_kt, ks * 2048), desc_add(d_tpp, ks * 32), ID_WU, ks > 0);
+            mma_commit(cx.bar(B_W_DONE));
+        }
+        __syncwarp();
     }
 }
 
@@ -314,39 +352,49 @@ __device__ void role_mma_chain(const Ctx& cx, const TcParams& prm)
         cx.wait(B_FULL_V, j & 1u);
         tc_fence_after();
         // U^T = V^T T'^T -> ACC1 (free: the Delta epilogue of chunk j-1 came before that chunk's last MMAs)
-#pragma unroll 1
-        for (int ks = 0; ks < 4; ++ks)
-            mma_ss(cx.tmem + TM_ACC1, desc_add(d_v, ks * 2048), desc_add(d_tp, ks * 32), ID_WU, ks > 0);
-        mma_commit(cx.bar(B_U_DONE));
+        if (elect_one()) {
+#pragma unroll
+            for (int ks = 0; ks < 4; ++ks)
+                mma_ss(cx.tmem + TM_ACC1, desc_add(d_v, ks * 2048), desc_add(d_tp, ks * 32), ID_WU, ks > 0);
+            mma_commit(cx.bar(B_U_DONE));
+        }
+        __syncwarp();
         // state of the previous chunk converted (or, at a chain start, the previous chain's state read out)
         if (j >= 1) cx.wait(B_SBF_READY, (j - 1) & 1u);
         tc_fence_after();
-        if (!first) {
-#pragma unroll 1
+        if (!first && elect_one()) {
+#pragma unroll
             for (int ks = 0; ks < 8; ++ks)
                 mma_ts(cx.tmem + TM_ACC1, cx.tmem + TM_SBF + ks * 8, desc_add(d_wt, ks * 2048), ID_SW, 1u);
         }
+        __syncwarp();
         if (j >= 1) cx.wait(B_ACC23_FREE, (j - 1) & 1u);
         tc_fence_after();
-        if (!first) {
-#pragma unroll 1
-            for (int ks = 0; ks < 8; ++ks)
-                mma_ts(cx.tmem + TM_ACC2, cx.tmem + TM_SBF + ks * 8,
-                       desc_add(d_q, (ks >> 2) * 16384 + (ks & 3) * 32), ID_SQ, ks > 0);
+        if (elect_one()) {
+            if (!first) {
+#pragma unroll
+                for (int ks = 0; ks < 8; ++ks)
+                    mma_ts(cx.tmem + TM_ACC2, cx.tmem + TM_SBF + ks * 8,
+                           desc_add(d_q, (ks >> 2) * 16384 + (ks & 3) * 32), ID_SQ, ks > 0);
+            }
+            mma_commit(cx.bar(B_MMA1_DONE));
         }
-        mma_commit(cx.bar(B_MMA1_DONE));
+        __syncwarp();
         cx.wait(B_D_READY, j & 1u);
         tc_fence_after();
-#pragma unroll 1
-        for (int ks = 0; ks < 4; ++ks)
-            mma_ts(cx.tmem + TM_ACC3, cx.tmem + TM_DBF + ks * 8, desc_add(d_p, ks * 32), ID_DP, ks > 0);
-#pragma unroll 1
-        for (int ks = 0; ks < 4; ++ks)
-            mma_ts(cx.tmem + TM_S32, cx.tmem + TM_DPBF + ks * 8, desc_add(d_kn, ks * 2048), ID_DK,
-                   (!first || ks > 0) ? 1u : 0u);
-        mma_commit(cx.bar(B_MMA3_DONE));
-        mma_commit(cx.bar(B_KQ_FREE0 + j % 3u));
-        mma_commit(cx.bar(B_P_FREE0 + (j & 1u)));
+        if (elect_one()) {
+#pragma unroll
+            for (int ks = 0; ks < 4; ++ks)
+                mma_ts(cx.tmem + TM_ACC3, cx.tmem + TM_DBF + ks * 8, desc_add(d_p, ks * 32), ID_DP, ks > 0);
+#pragma unroll
+            for (int ks = 0; ks < 4; ++ks)
+                mma_ts(cx.tmem + TM_S32, cx.tmem + TM_DPBF + ks * 8, desc_add(d_kn, ks * 2048), ID_DK,
+                       (!first || ks > 0) ? 1u : 0u);
+            mma_commit(cx.bar(B_MMA3_DONE));
+            mma_commit(cx.bar(B_KQ_FREE0 + j % 3u));
+            mma_commit(cx.bar(B_P_FREE0 + (j & 1u)));
+        }
+        __syncwarp();
     }
 }
 
@@ -366,19 +414,28 @@ __device__ void role_pre(const Ctx& cx, const TcParams& prm, int wtid)
     ChunkCursor cc;
     cc.init(&p, prm.s.order);
     GDN_DBG(long long tt_[16] = {0}; long long tl_ = clock64(); int nch = 0;)
+    // log-decay and beta of a chunk are fetched one chunk ahead (two rows per lane; padding rows read as 0)
+    float g0 = 0.f, g1 = 0.f, b0 = 0.f, b1 = 0.f;
+    auto fetch_gb = [&](const ChunkCursor& c, float& rg0, float& rg1, float& rb0, float& rb1) {
+        const int r0 = c.row0(), nv = c.nvalid();
+        const bool ok0 = lane < nv, ok1 = lane + 32 < nv;
+        rg0 = ok0 ? p.g[(size_t)(r0 + lane) * p.Hv + c.h] : 0.f;
+        rg1 = ok1 ? p.g[(size_t)(r0 + lane + 32) * p.Hv + c.h] : 0.f;
+        rb0 = ok0 ? p.beta[(size_t)(r0 + lane) * p.Hv + c.h] : 0.f;
+        rb1 = ok1 ? p.beta[(size_t)(r0 + lane + 32) * p.Hv + c.h] : 0.f;
+    };
+    if (cc.valid) fetch_gb(cc, g0, g1, b0, b1);
 #pragma unroll 1
-    for (uint32_t j = 0; cc.valid; ++j, cc.advance()) {
-        const int row0 = cc.row0(), nvalid = cc.nvalid(), h = cc.h;
+    for (uint32_t j = 0; cc.valid; ++j) {
         Decay& dc = misc->decay[j & 3u];
+        ChunkCursor cn = cc;
+        cn.advance();
+        float ng0 = 0.f, ng1 = 0.f, nb0 = 0.f, nb1 = 0.f;
+        if (cn.valid) fetch_gb(cn, ng0, ng1, nb0, nb1);
         GDN_DBG(const bool dbg = prm.debug && blockIdx.x == 0 && cc.r == 0 && cc.c < 2;
                 float* dbase = prm.debug + cc.c * DBG_STRIDE;)
 
         // ---- decay scan: every warp scans the 64 log-decays (two per lane); warp 0 publishes ------------
-        const bool ok0 = lane < nvalid, ok1 = lane + 32 < nvalid;
-        const float g0 = ok0 ? p.g[(size_t)(row0 + lane) * p.Hv + h] : 0.f;
-        const float g1 = ok1 ? p.g[(size_t)(row0 + lane + 32) * p.Hv + h] : 0.f;
-        const float b0 = ok0 ? p.beta[(size_t)(row0 + lane) * p.Hv + h] : 0.f;
-        const float b1 = ok1 ? p.beta[(size_t)(row0 + lane + 32) * p.Hv + h] : 0.f;
         float G0 = g0 * kLog2e, G1 = g1 * kLog2e;
 #pragma unroll
         for (int off = 1; off < 32; off <<= 1) {
@@ -529,6 +586,7 @@ __device__ void role_pre(const Ctx& cx, const TcParams& prm, int wtid)
         // ---- T'' = X diag(beta e^G) (operand of the W^T MMA), T' = X diag(beta) (operand of the U^T MMA) ----
         // T' is single-buffered: the U^T MMA of chunk j-1 must have read it
         if (j >= 1) cx.wait(B_U_DONE, (j - 1) & 1u);
+        GDN_T(9);
         {
             const int tt = wtid >> 2, q = wtid & 3, c0 = 16 * q;      // row, 16-column quarter
             uint32_t w1[8], w2[8];
@@ -551,8 +609,10 @@ __device__ void role_pre(const Ctx& cx, const TcParams& prm, int wtid)
             *reinterpret_cast<uint4*>(cx.sm + SM_TPP + o0) = make_uint4(w2[0], w2[1], w2[2], w2[3]);
             *reinterpret_cast<uint4*>(cx.sm + SM_TPP + o1) = make_uint4(w2[4], w2[5], w2[6], w2[7]);
         }
+        GDN_T(10);
         fence_proxy_async_smem();
-        mbar_arrive(cx.bar(B_TPP_READY));
+        GDN_T(11);
+        warp_arrive(cx.bar(B_TPP_READY), lane);
         GDN_T(6);
 
         // ---- W^T epilogue: bf16 rows [dk][t] as the N-major operand of the S0 W^T MMA ----------------------
@@ -588,11 +648,13 @@ __device__ void role_pre(const Ctx& cx, const TcParams& prm, int wtid)
             }
         }
         tc_fence_before();
-        mbar_arrive(cx.bar(B_WACC_READ));                  // the accumulator may take the next Gram tile
+        warp_arrive(cx.bar(B_WACC_READ), lane);                  // the accumulator may take the next Gram tile
         fence_proxy_async_smem();
-        mbar_arrive(cx.bar(B_PRE_DONE0 + (j & 1u)));
+        warp_arrive(cx.bar(B_PRE_DONE0 + (j & 1u)), lane);
         GDN_T(8);
         GDN_DBG(++nch;)
+        cc = cn;
+        g0 = ng0; g1 = ng1; b0 = nb0; b1 = nb1;
     }
 #ifdef GDN_TC_DEBUG
     if (prm.debug && blockIdx.x == 0 && wtid == 0 && nch > 0) {
@@ -684,7 +746,7 @@ __device__ void role_chain(const Ctx& cx, const TcParams& prm, int wtid)
             }
             tmem_st_wait();
             tc_fence_before();
-            mbar_arrive(cx.bar(B_D_READY));
+            warp_arrive(cx.bar(B_D_READY), lane);
             GDN_T(2);
 
             // ---- state: bf16 copy for the next chunk's MMAs + pre-scaling, or the final state ----------------
@@ -695,8 +757,10 @@ __device__ void role_chain(const Ctx& cx, const TcParams& prm, int wtid)
             for (int g = 0; g < 4; ++g) {
                 const int c0 = 64 * hf + 16 * g;
                 uint32_t acc[16];
+                GDN_DBG(long long s0_ = clock64();)
                 tmem_ld16(tl + TM_S32 + c0, acc);
                 tmem_ld_wait();
+                GDN_DBG(long long s1_ = clock64();)
 #ifdef GDN_TC_DEBUG
                 if (dbg) {
 #pragma unroll
@@ -709,8 +773,14 @@ __device__ void role_chain(const Ctx& cx, const TcParams& prm, int wtid)
                     for (int i = 0; i < 8; ++i) pk[i] = pack_bf16x2(__uint_as_float(acc[2 * i]), __uint_as_float(acc[2 * i + 1]));
 #pragma unroll
                     for (int i = 0; i < 16; ++i) acc[i] = __float_as_uint(__uint_as_float(acc[i]) * eGCnext);
+                    GDN_DBG(long long s2_ = clock64();)
                     tmem_st8(tl + TM_SBF + (c0 >> 1), pk);
                     tmem_st16(tl + TM_S32 + c0, acc);
+                    GDN_DBG(long long s3_ = clock64();
+                            if (prm.debug && blockIdx.x == 0 && wtid == 0 && j == 10) {
+                                float* d = prm.debug + 2 * DBG_STRIDE + 32 + g * 4;
+                                d[0] = (float)(s1_ - s0_); d[1] = (float)(s2_ - s1_); d[2] = (float)(s3_ - s2_); d[3] = (float)(s0_ & 0xffffff);
+                            })
                 } else if (st_out) {
 #pragma unroll
                     for (int i = 0; i < 16; ++i) st_out[(c0 + i) * 128 + dv] = __uint_as_float(acc[i]);
@@ -718,7 +788,7 @@ __device__ void role_chain(const Ctx& cx, const TcParams& prm, int wtid)
             }
             tmem_st_wait();
             tc_fence_before();
-            mbar_arrive(cx.bar(B_SBF_READY));
+            warp_arrive(cx.bar(B_SBF_READY), lane);
             GDN_T(4);
 
             // ---- output epilogue: O^T = diag(e^G) (S0 Q^T) + Delta^T P^T, transposed through shared memory ----
@@ -758,7 +828,7 @@ __device__ void role_chain(const Ctx& cx, const TcParams& prm, int wtid)
                     }
                 }
                 tc_fence_before();
-                mbar_arrive(cx.bar(B_ACC23_FREE));
+                warp_arrive(cx.bar(B_ACC23_FREE), lane);
                 GDN_T(6);
                 if (og) {
                     wg_sync(2);
@@ -805,7 +875,7 @@ gdn_tc_kernel(const TcParams prm, const __grid_constant__ CUtensorMap tm_q,
         for (int i = 0; i < NUM_BARS; ++i) {
             const bool wg_bar = i == B_WACC_READ || i == B_TPP_READY || i == B_PRE_DONE0 || i == B_PRE_DONE1 ||
                                 i == B_D_READY || i == B_SBF_READY || i == B_ACC23_FREE;
-            mbar_init(cx.bar(i), wg_bar ? (uint32_t)kWgThreads : 1u);
+            mbar_init(cx.bar(i), wg_bar ? (uint32_t)(kWgThreads / 32) : 1u);
         }
         fence_mbar_init();
         cx.misc->abort = 0u;
@@ -816,17 +886,26 @@ gdn_tc_kernel(const TcParams prm, const __grid_constant__ CUtensorMap tm_q,
     tc_fence_after();
     cx.tmem = cx.misc->tmem_base;
 
+#ifdef GDN_TC_PROFILE
+    cx.prof_init();
+#endif
     if (warp == 0) {
-        if (lane == 0) role_producer(cx, prm, &tm_q, &tm_k, &tm_v);
+        role_producer(cx, prm, &tm_q, &tm_k, &tm_v);
     } else if (warp == 1) {
-        if (lane == 0) role_mma_chain(cx, prm);
+        role_mma_chain(cx, prm);
     } else if (warp == 2) {
-        if (lane == 0) role_mma_pre(cx, prm);
+        role_mma_pre(cx, prm);
     } else if (warp >= 4 && warp < 12) {
         role_pre(cx, prm, tid - 128);
     } else if (warp >= 12) {
         role_chain(cx, prm, tid - 384);
     }
+#ifdef GDN_TC_PROFILE
+    if (prm.debug && blockIdx.x == 0 && lane == 0 && (warp < 3 || warp == 4 || warp == 12)) {
+        const int slot = warp < 3 ? warp : (warp == 4 ? 3 : 4);
+        cx.prof_dump(prm.debug + slot * 32);
+    }
+#endif
 
     tc_fence_before();
     __syncthreads();
@@ -875,7 +954,7 @@ float* g_debug_buffer = nullptr;
 
 }  // namespace
 
-#ifdef GDN_TC_DEBUG
+#if defined(GDN_TC_DEBUG) || defined(GDN_TC_PROFILE)
 extern "C" GDN_API void gdn_debug_set_buffer(float* dev_ptr) { g_debug_buffer = dev_ptr; }
 #endif
 
