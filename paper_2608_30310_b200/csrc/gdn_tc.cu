@@ -9,7 +9,7 @@
 //   Gram  = [K;Q] K^T                        (MMA, 128 x 64: rows 0-63 K K^T, rows 64-127 Q K^T)
 //   A     = strict_lower(beta_t Gam (K K^T)),  P = lower_incl(Gam (Q K^T))
 //   X     = (I + A)^-1                        (16 x 16 diagonal blocks by substitution in fp32, block
-//                                              merges on mma.sync tf32)
+//                                              merges on mma.sync bf16 with ldmatrix-fed fragments)
 //   T'    = X diag(beta),  T'' = X diag(beta e^G)
 //   W^T   = K^T T''^T                         (MMA, 128(dk) x 64)
 //   Dl^T  = V^T T'^T - S0 W^T                 (two MMAs into one accumulator, second negated)
@@ -20,6 +20,8 @@
 //   warp 0      TMA producer: K/Q tiles two chunks ahead (3 slots), V one chunk ahead (1 slot)
 //   warp 1      issues the chain MMAs (U^T, S0 W^T, S0 Q^T, Dl^T P^T, state update)
 //   warp 2      issues the intra-chunk MMAs (Gram, W^T) for the next chunk
+//   warp 3      decay warp: loads g and beta up to three chunks ahead, scans the log-decay and publishes the
+//               per-chunk decay factors
 //   warps 4-11  "pre" group: decay scan, A / P, triangular solve, T', T'', W^T epilogue (chunk j+1)
 //   warps 12-19 "chain" group: Delta epilogue, state conversion, output epilogue (chunk j)
 // Each group has two warps per TMEM lane window (they split the columns), and every per-chunk loop is
@@ -38,9 +40,8 @@ namespace {
 
 using namespace ptx;
 
-constexpr int LDA = 68;                       // fp32 row stride of the A scratch (floats)
-constexpr int LDX = 72;                       // fp32 row stride of the X scratch
-constexpr int LDM = 40;                       // fp32 row stride of the merge scratch
+constexpr int LDA = 72;                       // bf16 row stride of the A and X scratch (144 B: conflict-free ldmatrix)
+constexpr int LDM = 40;                       // bf16 row stride of the merge scratch (80 B)
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr int kThreads = 640;      // 3 single-lane role warps (+1 idle), 8 pre warps, 8 chain warps
 constexpr int kWgThreads = 256;
@@ -54,21 +55,23 @@ constexpr uint32_t SM_TP = 131072;            // T'  [t][s] bf16                
 constexpr uint32_t SM_TPP = 139264;           // T'' [t][s] bf16                                             8 KB
 constexpr uint32_t SM_P = 147456;             // 2 x P [t][s] bf16                                          16 KB
 constexpr uint32_t SM_OST = 163840;           // O staging [t][dv] bf16                                     16 KB
-constexpr uint32_t SM_AF = 180224;            // A fp32 [64][LDA]
-constexpr uint32_t SM_XF = SM_AF + 64 * LDA * 4;   // X fp32 [64][LDX]
-constexpr uint32_t SM_MF = SM_XF + 64 * LDX * 4;   // merge scratch fp32 [32][LDM]
-constexpr uint32_t SM_MISC = SM_MF + 32 * LDM * 4;
+constexpr uint32_t SM_AH = 180224;            // A bf16 [64][LDA]
+constexpr uint32_t SM_XH = SM_AH + 64 * LDA * 2;   // X = (I + A)^-1 bf16 [64][LDA]
+constexpr uint32_t SM_MH = SM_XH + 64 * LDA * 2;   // merge scratch bf16 [32][LDM]
+constexpr uint32_t SM_MISC = ((SM_MH + 32 * LDM * 2 + 1023) / 1024) * 1024;
 
 enum Bar {
     B_FULL_KQ0 = 0, B_FULL_KQ1, B_FULL_KQ2, B_FULL_V, B_GRAM_DONE, B_W_DONE, B_U_DONE, B_MMA1_DONE,
     B_MMA3_DONE, B_KQ_FREE0, B_KQ_FREE1, B_KQ_FREE2, B_P_FREE0, B_P_FREE1, B_WACC_READ, B_TPP_READY,
-    B_PRE_DONE0, B_PRE_DONE1, B_D_READY, B_SBF_READY, B_ACC23_FREE, NUM_BARS
+    B_PRE_DONE0, B_PRE_DONE1, B_D_READY, B_SBF_READY, B_ACC23_FREE,
+    B_DECAY_READY0, B_DECAY_READY1, B_DECAY_READY2, B_DECAY_READY3,
+    B_DECAY_FREE0, B_DECAY_FREE1, B_DECAY_FREE2, B_DECAY_FREE3, NUM_BARS
 };
 
 // G2 = log2(e) * cumulative log-decay; bE = beta e^G; eG = e^G; eRest = e^{G_C - G}
-struct Decay { float G2[64], beta[64], bE[64], eG[64], eRest[64]; };
+struct Decay { float G2[64], beta[64], bE[64], eG[64], eRest[64]; float eGC; float pad[3]; };
 struct Misc {
-    Decay decay[4];                    // per-chunk decay factors, ring of 4 (pre writes, chain reads)
+    Decay decay[4];                    // per-chunk decay factors, ring of 4 (decay warp writes; pre and chain read)
     unsigned long long bars[NUM_BARS];
     uint32_t tmem_base;
     volatile uint32_t abort;
@@ -103,9 +106,14 @@ struct TcParams {
 #ifdef GDN_TC_DEBUG
 constexpr int DBG_STRIDE = 61440;
 #define GDN_DBG(x) x
-#define GDN_T(i) do { long long n_ = clock64(); tt_[i] += n_ - tl_; tl_ = n_; } while (0)
 #else
 #define GDN_DBG(x)
+#endif
+#if defined(GDN_TC_DEBUG) || defined(GDN_TC_PROFILE)
+#define GDN_TIMERS(x) x
+#define GDN_T(i) do { long long n_ = clock64(); tt_[i] += n_ - tl_; tl_ = n_; } while (0)
+#else
+#define GDN_TIMERS(x)
 #define GDN_T(i) do {} while (0)
 #endif
 
@@ -209,43 +217,66 @@ __device__ __forceinline__ void warp_arrive(uint32_t bar, int lane)
     __syncwarp();
     if (lane == 0) mbar_arrive(bar);
 }
-__device__ __forceinline__ uint32_t to_tf32(float x)
+// ---- small bf16 tensor-core helpers for the block merges of the triangular solve --------------------
+// Four 8x8 bf16 matrices of the 16 x 16 tile at (row0, col0) of a row-major shared-memory matrix:
+// plain -> A fragment {a0..a3}; transposed -> B fragments {b0, b1} of the two 8-column halves.
+__device__ __forceinline__ uint32_t tile_addr(uint32_t base, int ld, int row0, int col0, int lane)
 {
-    uint32_t r;
-    asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(r) : "f"(x));
-    return r;
+    return base + (uint32_t)(((row0 + (lane & 7) + ((lane >> 3) & 1) * 8) * ld + col0 + (lane >> 4) * 8) * 2);
 }
-__device__ __forceinline__ void mma_tf32(float (&c)[4], const uint32_t (&a)[4], const uint32_t (&b)[2])
+__device__ __forceinline__ void ldm_x4(uint32_t (&r)[4], uint32_t addr)
 {
-    asm volatile("mma.sync.aligned.m16n8k8.row.col.f32.tf32.tf32.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+__device__ __forceinline__ void ldm_x4_trans(uint32_t (&r)[4], uint32_t addr)
+{
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+__device__ __forceinline__ void mma_bf16(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1)
+{
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
                  : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
-                 : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b[0]), "r"(b[1]));
+                 : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
-// 16 x 8 tile of C += A[r0.., k0..k1) * B[k0..k1, n0..): A, B row-major fp32 (tf32-rounded) in shared memory
-__device__ __forceinline__ void tile_mma(float (&c)[4], const float* A, int lda, int r0, const float* B, int ldb,
-                                         int n0, int k0, int k1, int lane)
+// c (16 x 16, two 8-column halves) += A[ar0.., ak0..+16) * B[bk0..+16, bn0..+16)
+__device__ __forceinline__ void tile16_mma(float (&c)[2][4], uint32_t a_base, int lda, int ar0, int ak0,
+                                           uint32_t b_base, int ldb, int bk0, int bn0, int lane)
+{
+    uint32_t a[4], b[4];
+    ldm_x4(a, tile_addr(a_base, lda, ar0, ak0, lane));
+    ldm_x4_trans(b, tile_addr(b_base, ldb, bk0, bn0, lane));
+    mma_bf16(c[0], a, b[0], b[1]);
+    mma_bf16(c[1], a, b[2], b[3]);
+}
+// stores sign * c as bf16 at D[r0.., n0..+16) (row-major, ld elements)
+__device__ __forceinline__ void tile16_store(const float (&c)[2][4], float sign, uint8_t* D, int ld, int r0, int n0, int lane)
 {
     const int g = lane >> 2, t4 = lane & 3;
-    for (int k = k0; k < k1; k += 8) {
-        uint32_t a[4], b[2];
-        a[0] = __float_as_uint(A[(r0 + g) * lda + k + t4]);
-        a[1] = __float_as_uint(A[(r0 + g + 8) * lda + k + t4]);
-        a[2] = __float_as_uint(A[(r0 + g) * lda + k + t4 + 4]);
-        a[3] = __float_as_uint(A[(r0 + g + 8) * lda + k + t4 + 4]);
-        b[0] = __float_as_uint(B[(k + t4) * ldb + n0 + g]);
-        b[1] = __float_as_uint(B[(k + t4 + 4) * ldb + n0 + g]);
-        mma_tf32(c, a, b);
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+        *reinterpret_cast<uint32_t*>(D + ((r0 + g) * ld + n0 + 8 * h + 2 * t4) * 2) = pack_bf16x2(sign * c[h][0], sign * c[h][1]);
+        *reinterpret_cast<uint32_t*>(D + ((r0 + g + 8) * ld + n0 + 8 * h + 2 * t4) * 2) = pack_bf16x2(sign * c[h][2], sign * c[h][3]);
     }
 }
-// stores a 16 x 8 C tile (optionally negated), rounded to tf32, at D[r0.., n0..)
-__device__ __forceinline__ void tile_store(const float (&c)[4], float sign, float* D, int ldd, int r0, int n0, int lane)
+// 8 x 8 variants for the first merge level (two independent 8 x 8 problems per instruction pair)
+__device__ __forceinline__ void ldm_x2(uint32_t (&r)[2], uint32_t addr)
 {
-    const int g = lane >> 2, t4 = lane & 3;
-    float2 lo = make_float2(__uint_as_float(to_tf32(sign * c[0])), __uint_as_float(to_tf32(sign * c[1])));
-    float2 hi = make_float2(__uint_as_float(to_tf32(sign * c[2])), __uint_as_float(to_tf32(sign * c[3])));
-    *reinterpret_cast<float2*>(&D[(r0 + g) * ldd + n0 + 2 * t4]) = lo;
-    *reinterpret_cast<float2*>(&D[(r0 + g + 8) * ldd + n0 + 2 * t4]) = hi;
+    asm volatile("ldmatrix.sync.aligned.m8n8.x2.shared.b16 {%0,%1}, [%2];" : "=r"(r[0]), "=r"(r[1]) : "r"(addr));
 }
+__device__ __forceinline__ void ldm_x2_trans(uint32_t (&r)[2], uint32_t addr)
+{
+    asm volatile("ldmatrix.sync.aligned.m8n8.x2.trans.shared.b16 {%0,%1}, [%2];" : "=r"(r[0]), "=r"(r[1]) : "r"(addr));
+}
+// rows 0-7 of (A[8 x 8] * B[8 x 8]) in c[0], c[1] (row lane / 4, columns 2 (lane % 4) + {0, 1})
+__device__ __forceinline__ void mma_8x8(float (&c)[4], uint32_t a0, uint32_t b0)
+{
+    asm volatile("mma.sync.aligned.m16n8k8.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5}, {%6}, {%0,%1,%2,%3};"
+                 : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3]) : "r"(a0), "r"(0u), "r"(b0));
+}
+__device__ __forceinline__ float bf_lo(uint32_t w) { return __uint_as_float(w << 16); }
+__device__ __forceinline__ float bf_hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
 
 // ================================================================================================
 // warp 0: TMA producer
@@ -399,6 +430,46 @@ __device__ void role_mma_chain(const Ctx& cx, const TcParams& prm)
 }
 
 // ================================================================================================
+// warp 3: decay warp.  Runs up to three chunks ahead of the consumers (ring of four slots), which hides the
+// DRAM latency of the strided g / beta loads.
+// ================================================================================================
+__device__ void role_decay(const Ctx& cx, const TcParams& prm)
+{
+    const Problem& p = prm.p;
+    const int lane = threadIdx.x & 31;
+    ChunkCursor cc;
+    cc.init(&p, prm.s.order);
+#pragma unroll 1
+    for (uint32_t j = 0; cc.valid; ++j, cc.advance()) {
+        const int row0 = cc.row0(), nvalid = cc.nvalid(), h = cc.h;
+        const bool ok0 = lane < nvalid, ok1 = lane + 32 < nvalid;
+        const float g0 = ok0 ? p.g[(size_t)(row0 + lane) * p.Hv + h] : 0.f;
+        const float g1 = ok1 ? p.g[(size_t)(row0 + lane + 32) * p.Hv + h] : 0.f;
+        const float b0 = ok0 ? p.beta[(size_t)(row0 + lane) * p.Hv + h] : 0.f;
+        const float b1 = ok1 ? p.beta[(size_t)(row0 + lane + 32) * p.Hv + h] : 0.f;
+        float G0 = g0 * kLog2e, G1 = g1 * kLog2e;
+#pragma unroll
+        for (int off = 1; off < 32; off <<= 1) {
+            const float u0 = __shfl_up_sync(0xffffffffu, G0, off), u1 = __shfl_up_sync(0xffffffffu, G1, off);
+            if (lane >= off) { G0 += u0; G1 += u1; }
+        }
+        G1 += __shfl_sync(0xffffffffu, G0, 31);
+        const float GC = __shfl_sync(0xffffffffu, G1, 31);
+        const float e0 = ex2_approx(G0), e1 = ex2_approx(G1);
+        // the slot was last read by the chain group's output epilogue of chunk j - 4
+        if (j >= 4) cx.wait(B_DECAY_FREE0 + (j & 3u), ((j >> 2) - 1u) & 1u);
+        Decay& dc = cx.misc->decay[j & 3u];
+        dc.G2[lane] = G0; dc.G2[lane + 32] = G1;
+        dc.beta[lane] = b0; dc.beta[lane + 32] = b1;
+        dc.bE[lane] = b0 * e0; dc.bE[lane + 32] = b1 * e1;
+        dc.eG[lane] = e0; dc.eG[lane + 32] = e1;
+        dc.eRest[lane] = ex2_approx(GC - G0); dc.eRest[lane + 32] = ex2_approx(GC - G1);
+        if (lane == 0) dc.eGC = ex2_approx(GC);
+        warp_arrive(cx.bar(B_DECAY_READY0 + (j & 3u)), lane);
+    }
+}
+
+// ================================================================================================
 // warps 4-11: pre group (intra-chunk stage of the chunk one ahead of the chain)
 // ================================================================================================
 __device__ void role_pre(const Ctx& cx, const TcParams& prm, int wtid)
@@ -407,58 +478,26 @@ __device__ void role_pre(const Ctx& cx, const TcParams& prm, int wtid)
     const int lane = wtid & 31, pw = wtid >> 5;          // pw = 0..7
     const int w4 = pw & 3, hf = pw >> 2;                 // TMEM lane window, column half
     const uint32_t tl = cx.tmem + ((uint32_t)(w4 * 32) << 16);
-    float* AF = reinterpret_cast<float*>(cx.sm + SM_AF);
-    float* XF = reinterpret_cast<float*>(cx.sm + SM_XF);
-    float* MF = reinterpret_cast<float*>(cx.sm + SM_MF);
+    uint8_t* AH = cx.sm + SM_AH;
+    uint8_t* XH = cx.sm + SM_XH;
+    uint8_t* MH = cx.sm + SM_MH;
+    const uint32_t ah = cx.sb + SM_AH, xh = cx.sb + SM_XH, mh = cx.sb + SM_MH;
     Misc* misc = cx.misc;
     ChunkCursor cc;
     cc.init(&p, prm.s.order);
-    GDN_DBG(long long tt_[16] = {0}; long long tl_ = clock64(); int nch = 0;)
-    // log-decay and beta of a chunk are fetched one chunk ahead (two rows per lane; padding rows read as 0)
-    float g0 = 0.f, g1 = 0.f, b0 = 0.f, b1 = 0.f;
-    auto fetch_gb = [&](const ChunkCursor& c, float& rg0, float& rg1, float& rb0, float& rb1) {
-        const int r0 = c.row0(), nv = c.nvalid();
-        const bool ok0 = lane < nv, ok1 = lane + 32 < nv;
-        rg0 = ok0 ? p.g[(size_t)(r0 + lane) * p.Hv + c.h] : 0.f;
-        rg1 = ok1 ? p.g[(size_t)(r0 + lane + 32) * p.Hv + c.h] : 0.f;
-        rb0 = ok0 ? p.beta[(size_t)(r0 + lane) * p.Hv + c.h] : 0.f;
-        rb1 = ok1 ? p.beta[(size_t)(r0 + lane + 32) * p.Hv + c.h] : 0.f;
-    };
-    if (cc.valid) fetch_gb(cc, g0, g1, b0, b1);
+    GDN_TIMERS(long long tt_[16] = {0}; long long tl_ = clock64(); int nch = 0;)
 #pragma unroll 1
-    for (uint32_t j = 0; cc.valid; ++j) {
+    for (uint32_t j = 0; cc.valid; ++j, cc.advance()) {
         Decay& dc = misc->decay[j & 3u];
-        ChunkCursor cn = cc;
-        cn.advance();
-        float ng0 = 0.f, ng1 = 0.f, nb0 = 0.f, nb1 = 0.f;
-        if (cn.valid) fetch_gb(cn, ng0, ng1, nb0, nb1);
         GDN_DBG(const bool dbg = prm.debug && blockIdx.x == 0 && cc.r == 0 && cc.c < 2;
                 float* dbase = prm.debug + cc.c * DBG_STRIDE;)
-
-        // ---- decay scan: every warp scans the 64 log-decays (two per lane); warp 0 publishes ------------
-        float G0 = g0 * kLog2e, G1 = g1 * kLog2e;
-#pragma unroll
-        for (int off = 1; off < 32; off <<= 1) {
-            const float u0 = __shfl_up_sync(0xffffffffu, G0, off), u1 = __shfl_up_sync(0xffffffffu, G1, off);
-            if (lane >= off) { G0 += u0; G1 += u1; }
-        }
-        G1 += __shfl_sync(0xffffffffu, G0, 31);
-        if (pw == 0) {
-            const float GC = __shfl_sync(0xffffffffu, G1, 31);
-            const float e0 = ex2_approx(G0), e1 = ex2_approx(G1);
-            dc.G2[lane] = G0; dc.G2[lane + 32] = G1;
-            dc.beta[lane] = b0; dc.beta[lane + 32] = b1;
-            dc.bE[lane] = b0 * e0; dc.bE[lane + 32] = b1 * e1;
-            dc.eG[lane] = e0; dc.eG[lane + 32] = e1;
-            dc.eRest[lane] = ex2_approx(GC - G0); dc.eRest[lane + 32] = ex2_approx(GC - G1);
-        }
+        cx.wait(B_DECAY_READY0 + (j & 3u), (j >> 2) & 1u);     // decay factors of this chunk are published
         // this thread's row of the Gram tile: lane windows 0,1 hold K K^T rows, 2,3 hold Q K^T rows
         const int t = ((w4 & 1) << 5) + lane;
         const bool isA = w4 < 2;
-        const float G2t = (w4 & 1) ? G1 : G0;
-        const float rowscale = isA ? ((w4 & 1) ? b1 : b0) : 1.f;
+        const float G2t = dc.G2[t];
+        const float rowscale = isA ? dc.beta[t] : 1.f;
         const int t_lim = isA ? t : t + 1;               // keep columns s < t_lim
-        wg_sync(1);                                       // decay arrays visible
         GDN_T(0);
 
         // ---- Gram tile -> A (fp32 scratch) and P (bf16 operand), 16 columns at a time ----------------------
@@ -501,12 +540,16 @@ __device__ void role_pre(const Ctx& cx, const TcParams& prm, int wtid)
                     }
                 }
                 if (isA) {
-                    float* arow = AF + t * LDA + c0;
+                    uint8_t* arow = AH + (t * LDA + c0) * 2;
 #pragma unroll
-                    for (int i = 0; i < 16; i += 4)
-                        *reinterpret_cast<float4*>(arow + i) = make_float4(
-                            __uint_as_float(to_tf32(vals[i])), __uint_as_float(to_tf32(vals[i + 1])),
-                            __uint_as_float(to_tf32(vals[i + 2])), __uint_as_float(to_tf32(vals[i + 3])));
+                    for (int c8 = 0; c8 < 2; ++c8) {
+                        uint4 u;
+                        u.x = pack_bf16x2(vals[c8 * 8 + 0], vals[c8 * 8 + 1]);
+                        u.y = pack_bf16x2(vals[c8 * 8 + 2], vals[c8 * 8 + 3]);
+                        u.z = pack_bf16x2(vals[c8 * 8 + 4], vals[c8 * 8 + 5]);
+                        u.w = pack_bf16x2(vals[c8 * 8 + 6], vals[c8 * 8 + 7]);
+                        *reinterpret_cast<uint4*>(arow + c8 * 16) = u;
+                    }
                 } else {
 #pragma unroll
                     for (int c8 = 0; c8 < 2; ++c8) {
@@ -525,63 +568,96 @@ __device__ void role_pre(const Ctx& cx, const TcParams& prm, int wtid)
         GDN_T(2);
 
         // ---- X = (I + A)^-1 ----------------------------------------------------------------------------
-        // level 0: the four 16 x 16 diagonal blocks by forward substitution; warps 0 and 1 take two blocks
-        // each (lane & 15 owns a column of block 2 pw + (lane >> 4))
+        // warps 0 and 1 each invert one 32 x 32 diagonal half without any cross-warp barrier:
+        //   level 0  : its four 8 x 8 diagonal blocks by forward substitution in fp32
+        //   level 0.5: 8 -> 16 merges, level 1: the 16 -> 32 merge X[hi][lo] = -X[hi][hi] (A[hi][lo] X[lo][lo]),
+        //              both on mma.sync with ldmatrix-fed bf16 fragments
         if (pw < 2) {
-            const int b = (2 * pw + (lane >> 4)) * 16, jj = lane & 15;
-            float x[16];
+            // level 0: four 8 x 8 diagonal blocks per warp (lane & 7 owns a column of block 4 pw + lane / 8)
+            {
+                const int bb = 4 * pw + (lane >> 3), b = 8 * bb, jj = lane & 7;
+                float x[8];
 #pragma unroll
-            for (int r = 0; r < 16; ++r) x[r] = (r == jj) ? 1.f : 0.f;
+                for (int r = 0; r < 8; ++r) x[r] = (r == jj) ? 1.f : 0.f;
 #pragma unroll
-            for (int r = 1; r < 16; ++r) {
-                float acc0 = 0.f, acc1 = 0.f;
+                for (int r = 1; r < 8; ++r) {
+                    const uint4 a4 = *reinterpret_cast<const uint4*>(AH + ((b + r) * LDA + b) * 2);
+                    const uint32_t wds[4] = {a4.x, a4.y, a4.z, a4.w};
+                    float acc0 = 0.f, acc1 = 0.f;
 #pragma unroll
-                for (int s2 = 0; s2 + 1 < r; s2 += 2) {
-                    acc0 = fmaf(AF[(b + r) * LDA + b + s2], x[s2], acc0);
-                    acc1 = fmaf(AF[(b + r) * LDA + b + s2 + 1], x[s2 + 1], acc1);
+                    for (int s2 = 0; s2 < r; ++s2) {
+                        const float a = (s2 & 1) ? bf_hi(wds[s2 >> 1]) : bf_lo(wds[s2 >> 1]);
+                        if (s2 & 1) acc1 = fmaf(a, x[s2], acc1); else acc0 = fmaf(a, x[s2], acc0);
+                    }
+                    x[r] = (r > jj) ? -(acc0 + acc1) : x[r];
                 }
-                if (r & 1) acc0 = fmaf(AF[(b + r) * LDA + b + r - 1], x[r - 1], acc0);
-                x[r] = (r > jj) ? -(acc0 + acc1) : x[r];
-            }
+                const int zc = (bb & 1) ? b - 8 : b + 8;      // the other 8 columns of this block's 16 x 16 parent
 #pragma unroll
-            for (int r = 0; r < 16; ++r) XF[(b + r) * LDX + b + jj] = __uint_as_float(to_tf32(x[r]));
+                for (int r = 0; r < 8; ++r) {
+                    *reinterpret_cast<__nv_bfloat16*>(XH + ((b + r) * LDA + b + jj) * 2) = __float2bfloat16_rn(x[r]);
+                    if (!(bb & 1)) *reinterpret_cast<uint16_t*>(XH + ((b + r) * LDA + zc + jj) * 2) = 0;   // upper-right 8 x 8
+                }
+            }
+            __syncwarp();
+            // level 0.5: inside each of this warp's two 16 x 16 blocks, X21 = -X22 (A21 X11) with 8 x 8 pieces
+            {
+                const int i = (lane >> 3) & 1, rr = lane & 7, b16 = 32 * pw + 16 * i;
+                const int g = lane >> 2, t4 = lane & 3;
+                uint32_t a[2], bx[2];
+                ldm_x2(a, ah + ((b16 + 8 + rr) * LDA + b16) * 2);                    // A21 of both blocks
+                ldm_x2_trans(bx, xh + ((b16 + rr) * LDA + b16) * 2);                  // X11 of both blocks
+                float m0[4] = {0.f, 0.f, 0.f, 0.f}, m1[4] = {0.f, 0.f, 0.f, 0.f};
+                mma_8x8(m0, a[0], bx[0]);
+                mma_8x8(m1, a[1], bx[1]);
+                // M_i at rows 16 pw + 8 i of the merge scratch, columns 0-7
+                *reinterpret_cast<uint32_t*>(MH + ((16 * pw + g) * LDM + 2 * t4) * 2) = pack_bf16x2(m0[0], m0[1]);
+                *reinterpret_cast<uint32_t*>(MH + ((16 * pw + 8 + g) * LDM + 2 * t4) * 2) = pack_bf16x2(m1[0], m1[1]);
+                __syncwarp();
+                uint32_t a2[2], bm[2];
+                ldm_x2(a2, xh + ((b16 + 8 + rr) * LDA + b16 + 8) * 2);               // X22 of both blocks
+                ldm_x2_trans(bm, mh + ((16 * pw + 8 * i + rr) * LDM) * 2);           // M of both blocks
+                float d0[4] = {0.f, 0.f, 0.f, 0.f}, d1[4] = {0.f, 0.f, 0.f, 0.f};
+                mma_8x8(d0, a2[0], bm[0]);
+                mma_8x8(d1, a2[1], bm[1]);
+                const int c0b = 32 * pw, c1b = 32 * pw + 16;
+                *reinterpret_cast<uint32_t*>(XH + ((c0b + 8 + g) * LDA + c0b + 2 * t4) * 2) = pack_bf16x2(-d0[0], -d0[1]);
+                *reinterpret_cast<uint32_t*>(XH + ((c1b + 8 + g) * LDA + c1b + 2 * t4) * 2) = pack_bf16x2(-d1[0], -d1[1]);
+            }
+            __syncwarp();
+            const int lo = 32 * pw, hi = 32 * pw + 16;
+            float m[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
+            tile16_mma(m, ah, LDA, hi, lo, xh, LDA, lo, lo, lane);               // A[hi][lo] X[lo][lo]
+            tile16_store(m, 1.f, MH, LDM, 16 * pw, 0, lane);
+            __syncwarp();
+            float d[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
+            tile16_mma(d, xh, LDA, hi, hi, mh, LDM, 16 * pw, 0, lane);           // X[hi][hi] M
+            tile16_store(d, -1.f, XH, LDA, hi, lo, lane);
         }
         wg_sync(1);
         GDN_T(3);
-        // level 1: X[2p+1][2p] = -X[2p+1][2p+1] (A[2p+1][2p] X[2p][2p]); warps 0-3 -> (pair p, 8-column half)
+        // level 2: X[32:64][0:32] = -X22 (A21 X11); warps 0-3 take one 16 x 16 tile (mt, nt) each
         {
-            const int pr = (pw >> 1) & 1, nh = pw & 1, rb = 32 * pr + 16, cb0 = 32 * pr;
+            const int mt = (pw >> 1) & 1, nt = pw & 1;
             if (pw < 4) {
-                float c4[4] = {0.f, 0.f, 0.f, 0.f};
-                tile_mma(c4, AF + cb0, LDA, rb, XF + cb0 * LDX + cb0, LDX, 8 * nh, 0, 16, lane);
-                tile_store(c4, 1.f, MF, LDM, 16 * pr, 8 * nh, lane);
+                float m[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
+                // X11 is lower triangular: block column nt starts at block row nt
+                for (int kb = nt; kb < 2; ++kb)
+                    tile16_mma(m, ah, LDA, 32 + 16 * mt, 16 * kb, xh, LDA, 16 * kb, 16 * nt, lane);
+                tile16_store(m, 1.f, MH, LDM, 16 * mt, 16 * nt, lane);
             }
             wg_sync(1);
             if (pw < 4) {
-                float d4[4] = {0.f, 0.f, 0.f, 0.f};
-                tile_mma(d4, XF + rb, LDX, rb, MF + 16 * pr * LDM, LDM, 8 * nh, 0, 16, lane);
-                tile_store(d4, -1.f, XF + cb0, LDX, rb, 8 * nh, lane);
+                float d[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
+                // X22 is lower triangular: block row mt ends at block column mt
+                for (int kb = 0; kb <= mt; ++kb)
+                    tile16_mma(d, xh, LDA, 32 + 16 * mt, 32 + 16 * kb, mh, LDM, 16 * kb, 16 * nt, lane);
+                tile16_store(d, -1.f, XH, LDA, 32 + 16 * mt, 16 * nt, lane);
             }
             wg_sync(1);
         }
         GDN_T(4);
-        // level 2: X[32:64][0:32] = -X22 (A21 X11); warp -> 16 x 8 output tile (mt, nt, nh)
-        {
-            const int mt = pw >> 2, nt = (pw >> 1) & 1, nh = pw & 1, n0 = 16 * nt + 8 * nh;
-            float c4[4] = {0.f, 0.f, 0.f, 0.f};
-            // X11 is lower triangular: columns of block nt start at row 16 nt
-            tile_mma(c4, AF, LDA, 32 + 16 * mt, XF, LDX, n0, 16 * nt, 32, lane);
-            tile_store(c4, 1.f, MF, LDM, 16 * mt, n0, lane);
-            wg_sync(1);
-            float d4[4] = {0.f, 0.f, 0.f, 0.f};
-            // X22 is lower triangular: row block mt ends at column 16 (mt + 1)
-            tile_mma(d4, XF + 32, LDX, 32 + 16 * mt, MF, LDM, n0, 0, 16 * (mt + 1), lane);
-            tile_store(d4, -1.f, XF, LDX, 32 + 16 * mt, n0, lane);
-            wg_sync(1);
-        }
-        GDN_T(5);
 #ifdef GDN_TC_DEBUG
-        if (dbg) for (int e = wtid; e < 4096; e += kWgThreads) dbase[8192 + e] = ((e & 63) <= (e >> 6)) ? XF[(e >> 6) * LDX + (e & 63)] : 0.f;
+        if (dbg) for (int e = wtid; e < 4096; e += kWgThreads) dbase[8192 + e] = ((e & 63) <= (e >> 6)) ? __bfloat162float(*reinterpret_cast<const __nv_bfloat16*>(XH + ((e >> 6) * LDA + (e & 63)) * 2)) : 0.f;
 #endif
         // ---- T'' = X diag(beta e^G) (operand of the W^T MMA), T' = X diag(beta) (operand of the U^T MMA) ----
         // T' is single-buffered: the U^T MMA of chunk j-1 must have read it
@@ -591,17 +667,18 @@ __device__ void role_pre(const Ctx& cx, const TcParams& prm, int wtid)
             const int tt = wtid >> 2, q = wtid & 3, c0 = 16 * q;      // row, 16-column quarter
             uint32_t w1[8], w2[8];
 #pragma unroll
-            for (int i4 = 0; i4 < 4; ++i4) {
-                const float4 xv = *reinterpret_cast<const float4*>(&XF[tt * LDX + c0 + 4 * i4]);
-                const float4 bv = *reinterpret_cast<const float4*>(&dc.beta[c0 + 4 * i4]);
-                const float4 ev = *reinterpret_cast<const float4*>(&dc.bE[c0 + 4 * i4]);
-                const int s0 = c0 + 4 * i4;
-                const float x0 = (s0 <= tt) ? xv.x : 0.f, x1 = (s0 + 1 <= tt) ? xv.y : 0.f;
-                const float x2 = (s0 + 2 <= tt) ? xv.z : 0.f, x3 = (s0 + 3 <= tt) ? xv.w : 0.f;
-                w1[2 * i4] = pack_bf16x2(x0 * bv.x, x1 * bv.y);
-                w1[2 * i4 + 1] = pack_bf16x2(x2 * bv.z, x3 * bv.w);
-                w2[2 * i4] = pack_bf16x2(x0 * ev.x, x1 * ev.y);
-                w2[2 * i4 + 1] = pack_bf16x2(x2 * ev.z, x3 * ev.w);
+            for (int c8 = 0; c8 < 2; ++c8) {
+                const uint4 xv = *reinterpret_cast<const uint4*>(XH + (tt * LDA + c0 + 8 * c8) * 2);
+                const uint32_t xw[4] = {xv.x, xv.y, xv.z, xv.w};
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const int s0 = c0 + 8 * c8 + 2 * e;
+                    const float2 bv = *reinterpret_cast<const float2*>(&dc.beta[s0]);
+                    const float2 ev = *reinterpret_cast<const float2*>(&dc.bE[s0]);
+                    const float x0 = (s0 <= tt) ? bf_lo(xw[e]) : 0.f, x1 = (s0 + 1 <= tt) ? bf_hi(xw[e]) : 0.f;
+                    w1[4 * c8 + e] = pack_bf16x2(x0 * bv.x, x1 * bv.y);
+                    w2[4 * c8 + e] = pack_bf16x2(x0 * ev.x, x1 * ev.y);
+                }
             }
             const uint32_t o0 = tt * 128 + (((2 * q) ^ (tt & 7)) << 4), o1 = tt * 128 + (((2 * q + 1) ^ (tt & 7)) << 4);
             *reinterpret_cast<uint4*>(cx.sm + SM_TP + o0) = make_uint4(w1[0], w1[1], w1[2], w1[3]);
@@ -652,13 +729,17 @@ __device__ void role_pre(const Ctx& cx, const TcParams& prm, int wtid)
         fence_proxy_async_smem();
         warp_arrive(cx.bar(B_PRE_DONE0 + (j & 1u)), lane);
         GDN_T(8);
-        GDN_DBG(++nch;)
-        cc = cn;
-        g0 = ng0; g1 = ng1; b0 = nb0; b1 = nb1;
+        GDN_TIMERS(++nch;)
     }
 #ifdef GDN_TC_DEBUG
     if (prm.debug && blockIdx.x == 0 && wtid == 0 && nch > 0) {
         float* d = prm.debug + 2 * DBG_STRIDE;
+        d[0] = (float)nch;
+        for (int i = 0; i < 12; ++i) d[1 + i] = (float)tt_[i] / nch;
+    }
+#elif defined(GDN_TC_PROFILE)
+    if (prm.debug && blockIdx.x == 0 && wtid == 0 && nch > 0) {
+        float* d = prm.debug + 5 * 32;
         d[0] = (float)nch;
         for (int i = 0; i < 12; ++i) d[1 + i] = (float)tt_[i] / nch;
     }
@@ -678,7 +759,7 @@ __device__ void role_chain(const Ctx& cx, const TcParams& prm, int wtid)
     Misc* misc = cx.misc;
     __nv_bfloat16* __restrict__ og = reinterpret_cast<__nv_bfloat16*>(p.out_o);
     const uint32_t num_items = (uint32_t)p.num_seqs * (uint32_t)p.Hv;
-    GDN_DBG(long long tt_[16] = {0}; long long tl_ = clock64(); int nch = 0;)
+    GDN_TIMERS(long long tt_[16] = {0}; long long tl_ = clock64(); int nch = 0;)
 
     uint32_t j = 0;
 #pragma unroll 1
@@ -701,17 +782,6 @@ __device__ void role_chain(const Ctx& cx, const TcParams& prm, int wtid)
             const bool first = c == 0, last = c == nchunks - 1;
             const Decay& dc = misc->decay[j & 3u];
             GDN_DBG(const bool dbg = prm.debug && blockIdx.x == 0 && r == 0 && c < 2; float* dbase = prm.debug + c * DBG_STRIDE;)
-
-            // total log-decay of the next chunk (scales the carried state ahead of its update MMA)
-            float eGCnext = 1.f;
-            if (!last) {
-                const int nrow0 = row0 + 64, nnv = min(64, row_end - nrow0);
-                float gs = (lane < nnv ? p.g[(size_t)(nrow0 + lane) * p.Hv + h] : 0.f) +
-                           (lane + 32 < nnv ? p.g[(size_t)(nrow0 + lane + 32) * p.Hv + h] : 0.f);
-#pragma unroll
-                for (int off = 16; off > 0; off >>= 1) gs += __shfl_xor_sync(0xffffffffu, gs, off);
-                eGCnext = ex2_approx(gs * kLog2e);
-            }
 
             // ---- Delta epilogue: bf16 Delta^T and decayed Delta'^T as TMEM A operands ----------------------
             cx.wait(B_PRE_DONE0 + (j & 1u), (j >> 1) & 1u);      // decay factors of this chunk are published
@@ -750,6 +820,12 @@ __device__ void role_chain(const Ctx& cx, const TcParams& prm, int wtid)
             GDN_T(2);
 
             // ---- state: bf16 copy for the next chunk's MMAs + pre-scaling, or the final state ----------------
+            // total decay of the next chunk scales the carried state ahead of that chunk's update MMA
+            float eGCnext = 1.f;
+            if (!last) {
+                cx.wait(B_DECAY_READY0 + ((j + 1) & 3u), ((j + 1) >> 2) & 1u);
+                eGCnext = misc->decay[(j + 1) & 3u].eGC;
+            }
             cx.wait(B_MMA3_DONE, j & 1u);
             GDN_T(3);
             tc_fence_after();
@@ -829,6 +905,7 @@ __device__ void role_chain(const Ctx& cx, const TcParams& prm, int wtid)
                 }
                 tc_fence_before();
                 warp_arrive(cx.bar(B_ACC23_FREE), lane);
+                warp_arrive(cx.bar(B_DECAY_FREE0 + (j & 3u)), lane);    // last read of this chunk's decay factors
                 GDN_T(6);
                 if (og) {
                     wg_sync(2);
@@ -843,12 +920,18 @@ __device__ void role_chain(const Ctx& cx, const TcParams& prm, int wtid)
                 }
             }
             GDN_T(8);
-            GDN_DBG(++nch;)
+            GDN_TIMERS(++nch;)
         }
     }
 #ifdef GDN_TC_DEBUG
     if (prm.debug && blockIdx.x == 0 && wtid == 0 && nch > 0) {
         float* d = prm.debug + 2 * DBG_STRIDE + 16;
+        d[0] = (float)nch;
+        for (int i = 0; i < 12; ++i) d[1 + i] = (float)tt_[i] / nch;
+    }
+#elif defined(GDN_TC_PROFILE)
+    if (prm.debug && blockIdx.x == 0 && wtid == 0 && nch > 0) {
+        float* d = prm.debug + 6 * 32;
         d[0] = (float)nch;
         for (int i = 0; i < 12; ++i) d[1 + i] = (float)tt_[i] / nch;
     }
@@ -874,7 +957,8 @@ gdn_tc_kernel(const TcParams prm, const __grid_constant__ CUtensorMap tm_q,
     if (tid == 32) {
         for (int i = 0; i < NUM_BARS; ++i) {
             const bool wg_bar = i == B_WACC_READ || i == B_TPP_READY || i == B_PRE_DONE0 || i == B_PRE_DONE1 ||
-                                i == B_D_READY || i == B_SBF_READY || i == B_ACC23_FREE;
+                                i == B_D_READY || i == B_SBF_READY || i == B_ACC23_FREE ||
+                                (i >= B_DECAY_FREE0 && i <= B_DECAY_FREE3);
             mbar_init(cx.bar(i), wg_bar ? (uint32_t)(kWgThreads / 32) : 1u);
         }
         fence_mbar_init();
@@ -895,6 +979,8 @@ gdn_tc_kernel(const TcParams prm, const __grid_constant__ CUtensorMap tm_q,
         role_mma_chain(cx, prm);
     } else if (warp == 2) {
         role_mma_pre(cx, prm);
+    } else if (warp == 3) {
+        role_decay(cx, prm);
     } else if (warp >= 4 && warp < 12) {
         role_pre(cx, prm, tid - 128);
     } else if (warp >= 12) {
