@@ -51,18 +51,19 @@ constexpr uint32_t SM_KQ = 0;                 // 3 slots x {2 halves x [128 rows
 constexpr uint32_t KQ_SLOT = 32768;
 constexpr uint32_t SM_V = 98304;              // 2 halves x [64 rows] x 128 B                               16 KB
 constexpr uint32_t SM_WT = 114688;            // W^T [dk][t] bf16, 128 rows x 128 B                          16 KB
-constexpr uint32_t SM_TP = 131072;            // T'  [t][s] bf16                                             8 KB
-constexpr uint32_t SM_TPP = 139264;           // T'' [t][s] bf16                                             8 KB
-constexpr uint32_t SM_P = 147456;             // 2 x P [t][s] bf16                                          16 KB
-constexpr uint32_t SM_OST = 163840;           // O staging [t][dv] bf16                                     16 KB
-constexpr uint32_t SM_AH = 180224;            // A bf16 [64][LDA]
+constexpr uint32_t SM_TP = 131072;            // 2 x T'  [t][s] bf16                                        16 KB
+constexpr uint32_t SM_TPP = 147456;           // T'' [t][s] bf16                                             8 KB
+constexpr uint32_t SM_P = 155648;             // 3 x P [t][s] bf16                                          24 KB
+constexpr uint32_t SM_OST = 180224;           // O staging [t][dv] bf16                                     16 KB
+constexpr uint32_t SM_AH = 196608;            // A bf16 [64][LDA]
 constexpr uint32_t SM_XH = SM_AH + 64 * LDA * 2;   // X = (I + A)^-1 bf16 [64][LDA]
 constexpr uint32_t SM_MH = SM_XH + 64 * LDA * 2;   // merge scratch bf16 [32][LDM]
 constexpr uint32_t SM_MISC = ((SM_MH + 32 * LDM * 2 + 1023) / 1024) * 1024;
 
 enum Bar {
     B_FULL_KQ0 = 0, B_FULL_KQ1, B_FULL_KQ2, B_FULL_V, B_GRAM_DONE, B_W_DONE, B_U_DONE, B_MMA1_DONE,
-    B_MMA3_DONE, B_KQ_FREE0, B_KQ_FREE1, B_KQ_FREE2, B_P_FREE0, B_P_FREE1, B_WACC_READ, B_TPP_READY,
+    B_MMA3_DONE, B_KQ_FREE0, B_KQ_FREE1, B_KQ_FREE2, B_P_FREE0, B_P_FREE1, B_P_FREE2, B_TP_FREE0, B_TP_FREE1,
+    B_GRAM_READ, B_WACC_READ, B_TPP_READY,
     B_PRE_DONE0, B_PRE_DONE1, B_D_READY, B_SBF_READY, B_ACC23_FREE,
     B_DECAY_READY0, B_DECAY_READY1, B_DECAY_READY2, B_DECAY_READY3,
     B_DECAY_FREE0, B_DECAY_FREE1, B_DECAY_FREE2, B_DECAY_FREE3, NUM_BARS
@@ -86,9 +87,13 @@ constexpr uint32_t TM_SBF = 128;    // bf16 copy of the chunk-start state, 64 co
 constexpr uint32_t TM_ACC1 = 192;   // Delta^T accumulator (U^T - S0 W^T), 64 columns
 constexpr uint32_t TM_ACC2 = 256;   // S0 Q^T, 64 columns
 constexpr uint32_t TM_ACC3 = 320;   // Delta^T P^T, 64 columns
-constexpr uint32_t TM_GRAM = 384;   // Gram accumulator, later W^T accumulator, 64 columns
-constexpr uint32_t TM_DBF = 448;    // Delta^T bf16, 32 columns
-constexpr uint32_t TM_DPBF = 480;   // (Delta diag(e^{G_C - G}))^T bf16, 32 columns
+constexpr uint32_t TM_GRAM = 384;   // Gram accumulator, 64 columns
+constexpr uint32_t TM_WACC = 448;   // W^T accumulator, 64 columns
+// The bf16 Delta operands reuse the columns of the bf16 state copy: the copy is dead once the MMAs that read
+// it have completed (which the Delta epilogue waits for), and it is rewritten only after the MMAs that read
+// the Delta operands have completed.
+constexpr uint32_t TM_DBF = 128;    // Delta^T bf16, 32 columns
+constexpr uint32_t TM_DPBF = 160;   // (Delta diag(e^{G_C - G}))^T bf16, 32 columns
 
 constexpr uint32_t ID_GRAM = idesc_bf16(128, 64, 0, 0, 0);    // [K;Q] (K-major) x K (K-major)
 constexpr uint32_t ID_WU = idesc_bf16(128, 64, 1, 0, 0);      // K^T or V^T (M-major) x T (K-major)
@@ -330,16 +335,14 @@ __device__ __forceinline__ uint64_t desc_add(uint64_t d, uint32_t bytes) { retur
 // ================================================================================================
 __device__ void role_mma_pre(const Ctx& cx, const TcParams& prm)
 {
-    ChunkCursor cc;
-    cc.init(&prm.p, prm.s.order);
+    ChunkCursor cg;                       // cursor of the Gram MMAs, one chunk ahead of the W^T MMAs
+    cg.init(&prm.p, prm.s.order);
     const uint64_t d_tpp = smem_desc_sw128(cx.sb + SM_TPP, 16, 1024);
-#pragma unroll 1
-    for (uint32_t j = 0; cc.valid; ++j, cc.advance()) {
-        const uint32_t slot = j % 3u, kq = cx.sb + SM_KQ + slot * KQ_SLOT;
-        const uint64_t d_kq = smem_desc_sw128(kq, 16, 1024);            // [K;Q] rows, K-major
-        const uint64_t d_kt = smem_desc_sw128(kq, 16384, 1024);         // K tile as M-major operand (K^T)
+    auto gram = [&](uint32_t j) {         // Gram(j): needs the K/Q tiles and the accumulator read by chunk j-1
+        const uint32_t slot = j % 3u;
+        const uint64_t d_kq = smem_desc_sw128(cx.sb + SM_KQ + slot * KQ_SLOT, 16, 1024);   // [K;Q] rows, K-major
         cx.wait(B_FULL_KQ0 + slot, (j / 3u) & 1u);
-        if (j >= 1) cx.wait(B_WACC_READ, (j - 1) & 1u);
+        if (j >= 1) cx.wait(B_GRAM_READ, (j - 1) & 1u);
         tc_fence_after();
         if (elect_one()) {
 #pragma unroll
@@ -350,16 +353,32 @@ __device__ void role_mma_pre(const Ctx& cx, const TcParams& prm)
             mma_commit(cx.bar(B_GRAM_DONE));
         }
         __syncwarp();
+    };
+    auto wmma = [&](uint32_t j) {         // W^T(j) = K^T T''^T: needs T''(j) and the accumulator read by chunk j-1
+        const uint64_t d_kt = smem_desc_sw128(cx.sb + SM_KQ + (j % 3u) * KQ_SLOT, 16384, 1024);   // K^T, M-major
         cx.wait(B_TPP_READY, j & 1u);
+        if (j >= 1) cx.wait(B_WACC_READ, (j - 1) & 1u);
         tc_fence_after();
         if (elect_one()) {
 #pragma unroll
             for (int ks = 0; ks < 4; ++ks)
-                mma_ss(cx.tmem + TM_GRAM, desc_add(d_kt, ks * 2048), desc_add(d_tpp, ks * 32), ID_WU, ks > 0);
+                mma_ss(cx.tmem + TM_WACC, desc_add(d_kt, ks * 2048), desc_add(d_tpp, ks * 32), ID_WU, ks > 0);
             mma_commit(cx.bar(B_W_DONE));
         }
         __syncwarp();
+    };
+    if (!cg.valid) return;
+    gram(0);
+    cg.advance();
+    uint32_t j = 0;
+#pragma unroll 1
+    for (;; ++j) {
+        if (j >= 1) wmma(j - 1);
+        if (!cg.valid) break;
+        gram(j + 1);
+        cg.advance();
     }
+    wmma(j);
 }
 
 // ================================================================================================
@@ -370,14 +389,14 @@ __device__ void role_mma_chain(const Ctx& cx, const TcParams& prm)
     ChunkCursor cc;
     cc.init(&prm.p, prm.s.order);
     const uint64_t d_v = smem_desc_sw128(cx.sb + SM_V, 8192, 1024);     // V tile as M-major operand (V^T)
-    const uint64_t d_tp = smem_desc_sw128(cx.sb + SM_TP, 16, 1024);
     const uint64_t d_wt = smem_desc_sw128(cx.sb + SM_WT, 16, 1024);     // W^T rows [dk][t], N-major operand
 #pragma unroll 1
     for (uint32_t j = 0; cc.valid; ++j, cc.advance()) {
         const uint32_t kq = cx.sb + SM_KQ + (j % 3u) * KQ_SLOT;
         const uint64_t d_q = smem_desc_sw128(kq + 8192, 16, 1024);      // Q rows, K-major
         const uint64_t d_kn = smem_desc_sw128(kq, 16384, 1024);         // K tile as N-major operand
-        const uint64_t d_p = smem_desc_sw128(cx.sb + SM_P + (j & 1u) * 8192, 16, 1024);
+        const uint64_t d_p = smem_desc_sw128(cx.sb + SM_P + (j % 3u) * 8192, 16, 1024);
+        const uint64_t d_tp = smem_desc_sw128(cx.sb + SM_TP + (j & 1u) * 8192, 16, 1024);
         const bool first = cc.first();
         cx.wait(B_PRE_DONE0 + (j & 1u), (j >> 1) & 1u);
         cx.wait(B_FULL_V, j & 1u);
@@ -388,6 +407,7 @@ __device__ void role_mma_chain(const Ctx& cx, const TcParams& prm)
             for (int ks = 0; ks < 4; ++ks)
                 mma_ss(cx.tmem + TM_ACC1, desc_add(d_v, ks * 2048), desc_add(d_tp, ks * 32), ID_WU, ks > 0);
             mma_commit(cx.bar(B_U_DONE));
+            mma_commit(cx.bar(B_TP_FREE0 + (j & 1u)));
         }
         __syncwarp();
         // state of the previous chunk converted (or, at a chain start, the previous chain's state read out)
@@ -423,7 +443,7 @@ __device__ void role_mma_chain(const Ctx& cx, const TcParams& prm)
                        (!first || ks > 0) ? 1u : 0u);
             mma_commit(cx.bar(B_MMA3_DONE));
             mma_commit(cx.bar(B_KQ_FREE0 + j % 3u));
-            mma_commit(cx.bar(B_P_FREE0 + (j & 1u)));
+            mma_commit(cx.bar(B_P_FREE0 + j % 3u));
         }
         __syncwarp();
     }
@@ -486,8 +506,41 @@ __device__ void role_pre(const Ctx& cx, const TcParams& prm, int wtid)
     ChunkCursor cc;
     cc.init(&p, prm.s.order);
     GDN_TIMERS(long long tt_[16] = {0}; long long tl_ = clock64(); int nch = 0;)
+    // W^T epilogue of chunk jw (warps 4-7, all 64 columns of their lane window): bf16 rows [dk][t] as the
+    // N-major operand of the S0 W^T MMA; completes the operand set of chunk jw
+    auto w_epilogue = [&](uint32_t jw) {
+        cx.wait(B_W_DONE, jw & 1u);
+        tc_fence_after();
+        // W^T is single-buffered: the S0 W^T MMA of chunk jw-1 must have read it
+        if (jw >= 1) cx.wait(B_MMA1_DONE, (jw - 1) & 1u);
+        const int drow = w4 * 32 + lane;                      // dk index = TMEM lane
+        uint8_t* wrow = cx.sm + SM_WT + drow * 128;
+#pragma unroll 1
+        for (int g = 0; g < 4; ++g) {
+            const int c0 = 16 * g;
+            uint32_t acc[16];
+            tmem_ld16(tl + TM_WACC + c0, acc);
+            tmem_ld_wait();
+#pragma unroll
+            for (int c8 = 0; c8 < 2; ++c8) {
+                uint4 u;
+                u.x = pack_bf16x2(__uint_as_float(acc[c8 * 8 + 0]), __uint_as_float(acc[c8 * 8 + 1]));
+                u.y = pack_bf16x2(__uint_as_float(acc[c8 * 8 + 2]), __uint_as_float(acc[c8 * 8 + 3]));
+                u.z = pack_bf16x2(__uint_as_float(acc[c8 * 8 + 4]), __uint_as_float(acc[c8 * 8 + 5]));
+                u.w = pack_bf16x2(__uint_as_float(acc[c8 * 8 + 6]), __uint_as_float(acc[c8 * 8 + 7]));
+                *reinterpret_cast<uint4*>(wrow + ((((c0 >> 3) + c8) ^ (drow & 7)) << 4)) = u;
+            }
+        }
+        tc_fence_before();
+        warp_arrive(cx.bar(B_WACC_READ), lane);            // the accumulator may take the next W^T tile
+        fence_proxy_async_smem();
+        warp_arrive(cx.bar(B_PRE_DONE0 + (jw & 1u)), lane);
+    };
+    auto solve_sync = [&]() { asm volatile("bar.sync 3, 128;" ::: "memory"); };
+    uint32_t j_total = 0;
 #pragma unroll 1
     for (uint32_t j = 0; cc.valid; ++j, cc.advance()) {
+        j_total = j + 1;
         Decay& dc = misc->decay[j & 3u];
         GDN_DBG(const bool dbg = prm.debug && blockIdx.x == 0 && cc.r == 0 && cc.c < 2;
                 float* dbase = prm.debug + cc.c * DBG_STRIDE;)
@@ -504,10 +557,10 @@ __device__ void role_pre(const Ctx& cx, const TcParams& prm, int wtid)
         cx.wait(B_GRAM_DONE, j & 1u);
         GDN_T(1);
         tc_fence_after();
-        // the P buffer of chunk j was last read by the MMAs of chunk j-2
-        if (j >= 2) cx.wait(B_P_FREE0 + (j & 1u), ((j >> 1) - 1u) & 1u);
+        // the P buffer of chunk j was last read by the MMAs of chunk j-3
+        if (j >= 3) cx.wait(B_P_FREE0 + j % 3u, ((j / 3u) - 1u) & 1u);
         {
-            uint8_t* prow = cx.sm + SM_P + (j & 1u) * 8192 + t * 128;
+            uint8_t* prow = cx.sm + SM_P + (j % 3u) * 8192 + t * 128;
 #pragma unroll 1
             for (int g = 0; g < 2; ++g) {
                 const int cb = 2 * hf + g, c0 = 16 * cb;
@@ -564,6 +617,7 @@ __device__ void role_pre(const Ctx& cx, const TcParams& prm, int wtid)
             }
         }
         tc_fence_before();
+        warp_arrive(cx.bar(B_GRAM_READ), lane);            // the accumulator may take the next Gram tile
         wg_sync(1);
         GDN_T(2);
 
@@ -572,6 +626,11 @@ __device__ void role_pre(const Ctx& cx, const TcParams& prm, int wtid)
         //   level 0  : its four 8 x 8 diagonal blocks by forward substitution in fp32
         //   level 0.5: 8 -> 16 merges, level 1: the 16 -> 32 merge X[hi][lo] = -X[hi][hi] (A[hi][lo] X[lo][lo]),
         //              both on mma.sync with ldmatrix-fed bf16 fragments
+        if (pw >= 4) {
+            // warps 4-7 (one per TMEM lane window) are not needed by the solve: they convert W^T of the
+            // previous chunk meanwhile
+            if (j >= 1) w_epilogue(j - 1);
+        }
         if (pw < 2) {
             // level 0: four 8 x 8 diagonal blocks per warp (lane & 7 owns a column of block 4 pw + lane / 8)
             {
@@ -633,7 +692,7 @@ __device__ void role_pre(const Ctx& cx, const TcParams& prm, int wtid)
             tile16_mma(d, xh, LDA, hi, hi, mh, LDM, 16 * pw, 0, lane);           // X[hi][hi] M
             tile16_store(d, -1.f, XH, LDA, hi, lo, lane);
         }
-        wg_sync(1);
+        if (pw < 4) solve_sync();
         GDN_T(3);
         // level 2: X[32:64][0:32] = -X22 (A21 X11); warps 0-3 take one 16 x 16 tile (mt, nt) each
         {
@@ -644,8 +703,8 @@ __device__ void role_pre(const Ctx& cx, const TcParams& prm, int wtid)
                 for (int kb = nt; kb < 2; ++kb)
                     tile16_mma(m, ah, LDA, 32 + 16 * mt, 16 * kb, xh, LDA, 16 * kb, 16 * nt, lane);
                 tile16_store(m, 1.f, MH, LDM, 16 * mt, 16 * nt, lane);
+                solve_sync();
             }
-            wg_sync(1);
             if (pw < 4) {
                 float d[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
                 // X22 is lower triangular: block row mt ends at block column mt
@@ -660,8 +719,8 @@ __device__ void role_pre(const Ctx& cx, const TcParams& prm, int wtid)
         if (dbg) for (int e = wtid; e < 4096; e += kWgThreads) dbase[8192 + e] = ((e & 63) <= (e >> 6)) ? __bfloat162float(*reinterpret_cast<const __nv_bfloat16*>(XH + ((e >> 6) * LDA + (e & 63)) * 2)) : 0.f;
 #endif
         // ---- T'' = X diag(beta e^G) (operand of the W^T MMA), T' = X diag(beta) (operand of the U^T MMA) ----
-        // T' is single-buffered: the U^T MMA of chunk j-1 must have read it
-        if (j >= 1) cx.wait(B_U_DONE, (j - 1) & 1u);
+        // the T' buffer of chunk j was last read by the U^T MMA of chunk j-2
+        if (j >= 2) cx.wait(B_TP_FREE0 + (j & 1u), ((j >> 1) - 1u) & 1u);
         GDN_T(9);
         {
             const int tt = wtid >> 2, q = wtid & 3, c0 = 16 * q;      // row, 16-column quarter
@@ -681,8 +740,9 @@ __device__ void role_pre(const Ctx& cx, const TcParams& prm, int wtid)
                 }
             }
             const uint32_t o0 = tt * 128 + (((2 * q) ^ (tt & 7)) << 4), o1 = tt * 128 + (((2 * q + 1) ^ (tt & 7)) << 4);
-            *reinterpret_cast<uint4*>(cx.sm + SM_TP + o0) = make_uint4(w1[0], w1[1], w1[2], w1[3]);
-            *reinterpret_cast<uint4*>(cx.sm + SM_TP + o1) = make_uint4(w1[4], w1[5], w1[6], w1[7]);
+            uint8_t* tp = cx.sm + SM_TP + (j & 1u) * 8192;
+            *reinterpret_cast<uint4*>(tp + o0) = make_uint4(w1[0], w1[1], w1[2], w1[3]);
+            *reinterpret_cast<uint4*>(tp + o1) = make_uint4(w1[4], w1[5], w1[6], w1[7]);
             *reinterpret_cast<uint4*>(cx.sm + SM_TPP + o0) = make_uint4(w2[0], w2[1], w2[2], w2[3]);
             *reinterpret_cast<uint4*>(cx.sm + SM_TPP + o1) = make_uint4(w2[4], w2[5], w2[6], w2[7]);
         }
@@ -692,45 +752,10 @@ __device__ void role_pre(const Ctx& cx, const TcParams& prm, int wtid)
         warp_arrive(cx.bar(B_TPP_READY), lane);
         GDN_T(6);
 
-        // ---- W^T epilogue: bf16 rows [dk][t] as the N-major operand of the S0 W^T MMA ----------------------
-        cx.wait(B_W_DONE, j & 1u);
-        GDN_T(7);
-        tc_fence_after();
-        // W^T is single-buffered: the S0 W^T MMA of chunk j-1 must have read it
-        if (j >= 1) cx.wait(B_MMA1_DONE, (j - 1) & 1u);
-        {
-            const int drow = w4 * 32 + lane;                      // dk index = TMEM lane
-            uint8_t* wrow = cx.sm + SM_WT + drow * 128;
-#pragma unroll 1
-            for (int g = 0; g < 2; ++g) {
-                const int c0 = 32 * hf + 16 * g;
-                uint32_t acc[16];
-                tmem_ld16(tl + TM_GRAM + c0, acc);
-                tmem_ld_wait();
-#ifdef GDN_TC_DEBUG
-                if (dbg) {
-#pragma unroll
-                    for (int i = 0; i < 16; ++i) dbase[12288 + drow * 64 + c0 + i] = __uint_as_float(acc[i]);
-                }
-#endif
-#pragma unroll
-                for (int c8 = 0; c8 < 2; ++c8) {
-                    uint4 u;
-                    u.x = pack_bf16x2(__uint_as_float(acc[c8 * 8 + 0]), __uint_as_float(acc[c8 * 8 + 1]));
-                    u.y = pack_bf16x2(__uint_as_float(acc[c8 * 8 + 2]), __uint_as_float(acc[c8 * 8 + 3]));
-                    u.z = pack_bf16x2(__uint_as_float(acc[c8 * 8 + 4]), __uint_as_float(acc[c8 * 8 + 5]));
-                    u.w = pack_bf16x2(__uint_as_float(acc[c8 * 8 + 6]), __uint_as_float(acc[c8 * 8 + 7]));
-                    *reinterpret_cast<uint4*>(wrow + ((((c0 >> 3) + c8) ^ (drow & 7)) << 4)) = u;
-                }
-            }
-        }
-        tc_fence_before();
-        warp_arrive(cx.bar(B_WACC_READ), lane);                  // the accumulator may take the next Gram tile
-        fence_proxy_async_smem();
-        warp_arrive(cx.bar(B_PRE_DONE0 + (j & 1u)), lane);
         GDN_T(8);
         GDN_TIMERS(++nch;)
     }
+    if (pw >= 4 && j_total > 0) w_epilogue(j_total - 1);
 #ifdef GDN_TC_DEBUG
     if (prm.debug && blockIdx.x == 0 && wtid == 0 && nch > 0) {
         float* d = prm.debug + 2 * DBG_STRIDE;
@@ -739,7 +764,7 @@ __device__ void role_pre(const Ctx& cx, const TcParams& prm, int wtid)
     }
 #elif defined(GDN_TC_PROFILE)
     if (prm.debug && blockIdx.x == 0 && wtid == 0 && nch > 0) {
-        float* d = prm.debug + 5 * 32;
+        float* d = prm.debug + 5 * 48;
         d[0] = (float)nch;
         for (int i = 0; i < 12; ++i) d[1 + i] = (float)tt_[i] / nch;
     }
@@ -931,7 +956,7 @@ __device__ void role_chain(const Ctx& cx, const TcParams& prm, int wtid)
     }
 #elif defined(GDN_TC_PROFILE)
     if (prm.debug && blockIdx.x == 0 && wtid == 0 && nch > 0) {
-        float* d = prm.debug + 6 * 32;
+        float* d = prm.debug + 6 * 48;
         d[0] = (float)nch;
         for (int i = 0; i < 12; ++i) d[1 + i] = (float)tt_[i] / nch;
     }
@@ -956,10 +981,11 @@ gdn_tc_kernel(const TcParams prm, const __grid_constant__ CUtensorMap tm_q,
     }
     if (tid == 32) {
         for (int i = 0; i < NUM_BARS; ++i) {
-            const bool wg_bar = i == B_WACC_READ || i == B_TPP_READY || i == B_PRE_DONE0 || i == B_PRE_DONE1 ||
-                                i == B_D_READY || i == B_SBF_READY || i == B_ACC23_FREE ||
-                                (i >= B_DECAY_FREE0 && i <= B_DECAY_FREE3);
-            mbar_init(cx.bar(i), wg_bar ? (uint32_t)(kWgThreads / 32) : 1u);
+            // arrivals per phase: one per warp of the arriving group (8), or of its W^T half (4)
+            const bool wg_bar = i == B_GRAM_READ || i == B_TPP_READY || i == B_D_READY || i == B_SBF_READY ||
+                                i == B_ACC23_FREE || (i >= B_DECAY_FREE0 && i <= B_DECAY_FREE3);
+            const bool half_bar = i == B_WACC_READ || i == B_PRE_DONE0 || i == B_PRE_DONE1;
+            mbar_init(cx.bar(i), wg_bar ? (uint32_t)(kWgThreads / 32) : half_bar ? 4u : 1u);
         }
         fence_mbar_init();
         cx.misc->abort = 0u;
@@ -989,7 +1015,7 @@ gdn_tc_kernel(const TcParams prm, const __grid_constant__ CUtensorMap tm_q,
 #ifdef GDN_TC_PROFILE
     if (prm.debug && blockIdx.x == 0 && lane == 0 && (warp < 3 || warp == 4 || warp == 12)) {
         const int slot = warp < 3 ? warp : (warp == 4 ? 3 : 4);
-        cx.prof_dump(prm.debug + slot * 32);
+        cx.prof_dump(prm.debug + slot * 48);
     }
 #endif
 
