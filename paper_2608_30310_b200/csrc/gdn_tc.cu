@@ -70,7 +70,8 @@ enum Bar {
 };
 
 // G2 = log2(e) * cumulative log-decay; bE = beta e^G; eG = e^G; eRest = e^{G_C - G}
-struct Decay { float G2[64], beta[64], bE[64], eG[64], eRest[64]; float eGC; float pad[3]; };
+// colf[s] = 2^(G2_31 - G2_s), s < 32: column factors of the purely off-diagonal quadrant of Gam
+struct Decay { float G2[64], beta[64], bE[64], eG[64], eRest[64], colf[32]; float eGC; float G2mid; float pad[2]; };
 struct Misc {
     Decay decay[4];                    // per-chunk decay factors, ring of 4 (decay warp writes; pre and chain read)
     unsigned long long bars[NUM_BARS];
@@ -484,7 +485,9 @@ __device__ void role_decay(const Ctx& cx, const TcParams& prm)
         dc.bE[lane] = b0 * e0; dc.bE[lane + 32] = b1 * e1;
         dc.eG[lane] = e0; dc.eG[lane + 32] = e1;
         dc.eRest[lane] = ex2_approx(GC - G0); dc.eRest[lane + 32] = ex2_approx(GC - G1);
-        if (lane == 0) dc.eGC = ex2_approx(GC);
+        const float G31 = __shfl_sync(0xffffffffu, G0, 31);
+        dc.colf[lane] = ex2_approx(G31 - G0);
+        if (lane == 0) { dc.eGC = ex2_approx(GC); dc.G2mid = G31; }
         warp_arrive(cx.bar(B_DECAY_READY0 + (j & 3u)), lane);
     }
 }
@@ -561,9 +564,13 @@ __device__ void role_pre(const Ctx& cx, const TcParams& prm, int wtid)
         if (j >= 3) cx.wait(B_P_FREE0 + j % 3u, ((j / 3u) - 1u) & 1u);
         {
             uint8_t* prow = cx.sm + SM_P + (j % 3u) * 8192 + t * 128;
+            // column blocks are dealt so that each warp of a lane window gets one block that touches the
+            // diagonal and one that does not: half 0 -> blocks {0, 2}, half 1 -> blocks {1, 3}
+            const bool lower_rows = (w4 & 1) != 0;             // rows 32-63
+            const float rowf = lower_rows ? ex2_approx(G2t - dc.G2mid) * rowscale : 0.f;
 #pragma unroll 1
             for (int g = 0; g < 2; ++g) {
-                const int cb = 2 * hf + g, c0 = 16 * cb;
+                const int cb = hf + 2 * g, c0 = 16 * cb;
                 if (c0 > ((w4 & 1) << 5) + 31) {          // block entirely above the diagonal (warp-uniform)
                     if (!isA) {
                         *reinterpret_cast<uint4*>(prow + (((2 * cb) ^ (t & 7)) << 4)) = make_uint4(0u, 0u, 0u, 0u);
@@ -581,15 +588,28 @@ __device__ void role_pre(const Ctx& cx, const TcParams& prm, int wtid)
                 }
 #endif
                 float vals[16];
+                if (lower_rows && cb < 2) {
+                    // every column precedes every row of this warp: Gam = rowf * colf, no mask, no exp
 #pragma unroll
-                for (int i4 = 0; i4 < 4; ++i4) {
-                    const float4 gs = *reinterpret_cast<const float4*>(&dc.G2[c0 + 4 * i4]);
-                    const float gss[4] = {gs.x, gs.y, gs.z, gs.w};
+                    for (int i4 = 0; i4 < 4; ++i4) {
+                        const float4 cf = *reinterpret_cast<const float4*>(&dc.colf[c0 + 4 * i4]);
+                        vals[4 * i4 + 0] = (rowf * cf.x) * __uint_as_float(acc[4 * i4 + 0]);
+                        vals[4 * i4 + 1] = (rowf * cf.y) * __uint_as_float(acc[4 * i4 + 1]);
+                        vals[4 * i4 + 2] = (rowf * cf.z) * __uint_as_float(acc[4 * i4 + 2]);
+                        vals[4 * i4 + 3] = (rowf * cf.w) * __uint_as_float(acc[4 * i4 + 3]);
+                    }
+                } else {
 #pragma unroll
-                    for (int e = 0; e < 4; ++e) {
-                        const int i = 4 * i4 + e;
-                        const float f = ex2_approx(fminf(G2t - gss[e], 0.f)) * rowscale;
-                        vals[i] = (c0 + i < t_lim) ? f * __uint_as_float(acc[i]) : 0.f;
+                    for (int i4 = 0; i4 < 4; ++i4) {
+                        const float4 gs = *reinterpret_cast<const float4*>(&dc.G2[c0 + 4 * i4]);
+                        const float gss[4] = {gs.x, gs.y, gs.z, gs.w};
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            const int i = 4 * i4 + e;
+                            // masked entries may overflow to inf / NaN before the select discards them
+                            const float f = ex2_approx(G2t - gss[e]) * rowscale;
+                            vals[i] = (c0 + i < t_lim) ? f * __uint_as_float(acc[i]) : 0.f;
+                        }
                     }
                 }
                 if (isA) {
