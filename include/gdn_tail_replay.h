@@ -64,7 +64,8 @@ typedef enum {
     GDN_ERR_UNSUPPORTED = -2,   /* head dims, chunk, dtype or kernel choice not built */
     GDN_ERR_WORKSPACE = -3,     /* workspace missing or smaller than gdn_workspace_size() */
     GDN_ERR_CUDA = -4,          /* a CUDA runtime / driver call failed */
-    GDN_ERR_TIMEOUT = -5        /* device-side bounded wait expired (status_word only) */
+    GDN_ERR_TIMEOUT = -5,       /* device-side bounded wait expired (status_word only) */
+    GDN_ERR_TOO_LARGE = -6      /* more requests than the built-in scratch of the no-allocation entry holds */
 } gdn_status;
 
 typedef enum { GDN_F32 = 0, GDN_BF16 = 1 } gdn_dtype;
@@ -119,6 +120,37 @@ GDN_API int32_t gdn_tail_replay(const gdn_desc* desc, const void* q, const void*
 GDN_API int32_t gdn_full_prefill(const gdn_desc* desc, const void* q, const void* k, const void* v,
                          const float* g, const float* beta, const int32_t* cu_tail_lens,
                          int32_t chunk, void* out_o, float* out_state);
+
+/*
+ * Tail replay for callers that have no device memory to hand over as workspace.  (The paper has no
+ * counterpart: this entry point exists for integration reasons only.)
+ *
+ * Who needs it: a serving process that reserved the whole HBM for its own cache pool at start-up and can
+ * neither spare a slice for a library nor risk a cudaMalloc in the middle of serving (it may fail outright,
+ * and it stalls every stream of the device while it runs); and callers that only hold raw pointers handed
+ * down from another runtime's allocator and have no allocator of their own to ask.
+ *
+ * It is gdn_tail_replay with the scheduler scratch (work counter + longest-first request order) taken from
+ * an array that is compiled into the library's device image instead of from desc->workspace, which is
+ * ignored together with desc->workspace_bytes.  The array is GDN_STATIC_SCRATCH_BYTES large and is held by
+ * every GPU that loads the library until the process exits.  Limits and rules:
+ *   - desc->num_seqs <= GDN_STATIC_SCRATCH_MAX_SEQS, otherwise GDN_ERR_TOO_LARGE (nothing is enqueued);
+ *   - device pointers only (desc->memory == GDN_MEM_DEVICE), otherwise GDN_ERR_UNSUPPORTED: staging host
+ *     buffers would need far more scratch than is built in;
+ *   - the first call on each device looks up the array's device address (with that device current) and
+ *     caches it; make that first call before starting any stream capture;
+ *   - the call itself allocates and frees nothing, on the host side of CUDA or on the device;
+ *   - every call on a device shares the one array and the array keeps the previous call's contents; the
+ *     scheduler kernel rewrites the counter and the part of the order list it uses before the forward
+ *     kernel reads them, so back-to-back calls on one stream are fine, but two calls that overlap on the
+ *     GPU (different streams, or different host threads without ordering) race on it and are not allowed.
+ * All other arguments, layouts, results and error codes are those of gdn_tail_replay.
+ */
+#define GDN_STATIC_SCRATCH_MAX_SEQS 4096
+#define GDN_STATIC_SCRATCH_BYTES (256 + 4 * GDN_STATIC_SCRATCH_MAX_SEQS)
+GDN_API int32_t gdn_tail_replay_static_scratch(const gdn_desc* desc, const void* q, const void* k, const void* v,
+                                               const float* g, const float* beta, const int32_t* cu_tail_lens,
+                                               int32_t chunk, void* out_o, float* out_state);
 
 /*
  * Replay-window length k = ceil(budget_frac * prefix_len) (paper, Method section); the

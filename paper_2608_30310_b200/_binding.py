@@ -53,7 +53,7 @@ def load_library():
     fwd_args = [dp, vp, vp, vp, vp, vp, vp, ctypes.c_int32, vp, vp]
     lib.gdn_workspace_size.restype = ctypes.c_size_t
     lib.gdn_workspace_size.argtypes = [dp]
-    for name in ("gdn_tail_replay", "gdn_full_prefill"):
+    for name in ("gdn_tail_replay", "gdn_full_prefill", "gdn_tail_replay_static_scratch"):
         fn = getattr(lib, name)
         fn.restype = ctypes.c_int32
         fn.argtypes = fwd_args
@@ -140,10 +140,13 @@ def _forward(fn_name, q, k, v, g, beta, cu_tail_lens, chunk, out_o, out_state, *
     desc.memory = GDN_MEM_HOST if host else GDN_MEM_DEVICE
     desc.kernel = kernel
     desc.init_state = _ptr(init_state)
-    need = int(lib.gdn_workspace_size(ctypes.byref(desc)))
-    if workspace is None:
-        workspace = Workspace(device="cuda" if host else q.device)
-    desc.workspace, desc.workspace_bytes = workspace.ensure(need)
+    if fn_name == "gdn_tail_replay_static_scratch":
+        desc.workspace, desc.workspace_bytes = None, 0          # ignored: the library's built-in scratch is used
+    else:
+        need = int(lib.gdn_workspace_size(ctypes.byref(desc)))
+        if workspace is None:
+            workspace = Workspace(device="cuda" if host else q.device)
+        desc.workspace, desc.workspace_bytes = workspace.ensure(need)
     desc.status_word = _ptr(status_word)
     if stream is None:
         stream = torch.cuda.current_stream()
@@ -164,6 +167,15 @@ def gdn_tail_replay(q, k, v, g, beta, cu_tail_lens, chunk, out_o, out_state, **k
     check.
     """
     return _forward("gdn_tail_replay", q, k, v, g, beta, cu_tail_lens, chunk, out_o, out_state, **kw)
+
+
+def gdn_tail_replay_static_scratch(q, k, v, g, beta, cu_tail_lens, chunk, out_o, out_state, **kw) -> int:
+    """``gdn_tail_replay`` for callers with no device memory to spare: the scheduler scratch comes from an
+    array built into the library instead of a workspace, and the call allocates nothing (this binding passes
+    no workspace and creates no tensor).  Device tensors only, at most 4096 requests per call, and calls
+    must not overlap on the GPU because they all share that one array.  Make the first call on a device
+    outside any stream capture: it looks up the array's address once."""
+    return _forward("gdn_tail_replay_static_scratch", q, k, v, g, beta, cu_tail_lens, chunk, out_o, out_state, **kw)
 
 
 def gdn_full_prefill(q, k, v, g, beta, cu_tail_lens, chunk, out_o, out_state, **kw) -> int:

@@ -2,9 +2,20 @@
 // Every step of the path itself runs in the kernels of sched.cu, gdn_simt.cu and gdn_tc.cu.
 #include <math.h>
 #include <string.h>
+#include <mutex>
 #include "common.cuh"
 
 namespace {
+
+// Built-in scheduler scratch of gdn_tail_replay_static_scratch: lives in the library's device image, one
+// copy per GPU that loads it.  In host code this name is only a handle for cudaGetSymbolAddress, never a
+// device address.
+static __device__ __align__(256) unsigned char g_static_scratch[GDN_STATIC_SCRATCH_BYTES];
+static_assert(GDN_STATIC_SCRATCH_BYTES == sizeof(gdn::SchedHeader) + sizeof(int32_t) * GDN_STATIC_SCRATCH_MAX_SEQS,
+              "built-in scratch = scheduler header + one order entry per request");
+constexpr int kMaxDevices = 64;
+void* g_static_scratch_addr[kMaxDevices] = {};
+std::mutex g_static_scratch_mutex;
 
 thread_local int g_last_launches = 0;
 
@@ -170,6 +181,33 @@ int32_t gdn_full_prefill(const gdn_desc* desc, const void* q, const void* k, con
     return forward(desc, q, k, v, g, beta, cu_tail_lens, chunk, out_o, out_state);
 }
 
+int32_t gdn_tail_replay_static_scratch(const gdn_desc* desc, const void* q, const void* k, const void* v,
+                                       const float* g, const float* beta, const int32_t* cu_tail_lens,
+                                       int32_t chunk, void* out_o, float* out_state)
+{
+    if (!desc) return GDN_ERR_INVALID_ARG;
+    if (desc->memory != GDN_MEM_DEVICE) return GDN_ERR_UNSUPPORTED;
+    if (desc->num_seqs > GDN_STATIC_SCRATCH_MAX_SEQS) return GDN_ERR_TOO_LARGE;
+    if (desc->num_seqs <= 0) return forward(desc, q, k, v, g, beta, cu_tail_lens, chunk, out_o, out_state);
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return GDN_ERR_CUDA;
+    void* scratch = nullptr;
+    {
+        // one-time set-up per device: resolve the array's address on the current device
+        std::lock_guard<std::mutex> lock(g_static_scratch_mutex);
+        if (!g_static_scratch_addr[dev]) {
+            void* addr = nullptr;
+            if (cudaGetSymbolAddress(&addr, g_static_scratch) != cudaSuccess || !addr) return GDN_ERR_CUDA;
+            g_static_scratch_addr[dev] = addr;
+        }
+        scratch = g_static_scratch_addr[dev];
+    }
+    gdn_desc d = *desc;
+    d.workspace = scratch;
+    d.workspace_bytes = GDN_STATIC_SCRATCH_BYTES;
+    return forward(&d, q, k, v, g, beta, cu_tail_lens, chunk, out_o, out_state);
+}
+
 int64_t tail_select(int64_t prefix_len, double budget_frac)
 {
     if (prefix_len < 0 || budget_frac != budget_frac || budget_frac < 0.0) return -1;
@@ -191,6 +229,7 @@ const char* gdn_status_string(int32_t status)
         case GDN_ERR_WORKSPACE: return "workspace missing or too small";
         case GDN_ERR_CUDA: return "CUDA call failed";
         case GDN_ERR_TIMEOUT: return "device-side wait timed out";
+        case GDN_ERR_TOO_LARGE: return "more requests than the built-in scratch holds";
         default: return "unknown status";
     }
 }
