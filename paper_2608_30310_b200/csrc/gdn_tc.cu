@@ -205,12 +205,10 @@ struct Ctx {
         if (misc->abort) return true;
         const uint64_t t0 = globaltimer_ns();
         for (uint32_t it = 0;; ++it) {
-            __nanosleep(40);                       // back off: spinning warps would steal issue slots
-            if (mbar_try_wait(b, parity)) return true;
-            if ((it & 63u) == 63u) {
-                if (misc->abort) return true;
-                if (globaltimer_ns() - t0 > 2000000000ull) { misc->abort = 1u; return true; }
-            }
+            // suspended in hardware until the phase completes (or ~20 us pass): no polling instructions
+            if (mbar_try_wait_hint(b, parity, 20000u)) return true;
+            if (misc->abort) return true;
+            if (globaltimer_ns() - t0 > 2000000000ull) { misc->abort = 1u; return true; }
         }
     }
 };
