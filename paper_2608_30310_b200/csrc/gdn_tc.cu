@@ -910,11 +910,12 @@ __device__ void role_chain(const Ctx& cx, const TcParams& prm, int wtid)
             warp_arrive(cx.bar(B_SBF_READY), lane);
             GDN_T(4);
 
-            // ---- output epilogue: O^T = diag(e^G) (S0 Q^T) + Delta^T P^T, transposed through shared memory ----
+            // ---- output epilogue: O^T = diag(e^G) (S0 Q^T) + Delta^T P^T -------------------------------------
+            // For a fixed token the 128 lanes hold 128 consecutive bf16 of out_o: each warp store writes 64
+            // contiguous bytes (two full sectors), so the outputs go straight from registers to global memory.
             {
-                __nv_bfloat16* ost = reinterpret_cast<__nv_bfloat16*>(cx.sm + SM_OST);
-                if (og) wg_sync(2);                            // previous chunk's staged tile fully drained
-                GDN_T(5);
+                __nv_bfloat16* obase = og ? og + ((size_t)row0 * p.Hv + h) * 128 + dv : nullptr;
+                const size_t ostride = (size_t)p.Hv * 128;
 #pragma unroll 1
                 for (int g = 0; g < 2; ++g) {
                     const int c0 = 32 * hf + 16 * g;
@@ -941,7 +942,7 @@ __device__ void role_chain(const Ctx& cx, const TcParams& prm, int wtid)
                                 const int i = 4 * i4 + e;
                                 float o = __uint_as_float(a3[i]);
                                 if (!first) o = fmaf(egs[e], __uint_as_float(a2[i]), o);
-                                ost[(c0 + i) * 128 + dv] = __float2bfloat16_rn(o);
+                                if (c0 + i < nvalid) obase[(size_t)(c0 + i) * ostride] = __float2bfloat16_rn(o);
                             }
                         }
                     }
@@ -950,17 +951,6 @@ __device__ void role_chain(const Ctx& cx, const TcParams& prm, int wtid)
                 warp_arrive(cx.bar(B_ACC23_FREE), lane);
                 warp_arrive(cx.bar(B_DECAY_FREE0 + (j & 3u)), lane);    // last read of this chunk's decay factors
                 GDN_T(6);
-                if (og) {
-                    wg_sync(2);
-                    GDN_T(7);
-                    const uint4* src = reinterpret_cast<const uint4*>(cx.sm + SM_OST);
-#pragma unroll
-                    for (int it = 0; it < 4; ++it) {
-                        const int idx = it * kWgThreads + wtid, row = idx >> 4, c16 = idx & 15;
-                        if (row < nvalid)
-                            *reinterpret_cast<uint4*>(reinterpret_cast<uint8_t*>(og) + (((size_t)(row0 + row) * p.Hv + h) * 256 + c16 * 16)) = src[idx];
-                    }
-                }
             }
             GDN_T(8);
             GDN_TIMERS(++nch;)
