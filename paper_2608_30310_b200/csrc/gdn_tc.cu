@@ -16,17 +16,21 @@
 //   O^T   = (S0 Q^T) diag(e^G) + Dl^T P^T     (two MMAs, combined in the epilogue)
 //   S     = e^{G_C} S0 + (Dl diag(e^{G_C - G}))^T K    (MMA accumulating onto the pre-scaled state)
 //
-// The CTA is warp-specialised and software-pipelined over the chunks of all chains it owns:
-//   warp 0      TMA producer: K/Q tiles two chunks ahead (3 slots), V one chunk ahead (1 slot)
-//   warp 1      issues the chain MMAs (U^T, S0 W^T, S0 Q^T, Dl^T P^T, state update)
-//   warp 2      issues the intra-chunk MMAs (Gram, W^T) for the next chunk
-//   warp 3      decay warp: loads g and beta up to three chunks ahead, scans the log-decay and publishes the
-//               per-chunk decay factors
-//   warps 4-11  "pre" group: decay scan, A / P, triangular solve, T', T'', W^T epilogue (chunk j+1)
-//   warps 12-19 "chain" group: Delta epilogue, state conversion, output epilogue (chunk j)
-// Each group has two warps per TMEM lane window (they split the columns), and every per-chunk loop is
-// kept rolled with 16-column TMEM accesses: straight-line code larger than the instruction caches runs
-// at a fraction of the issue rate, so the static footprint matters as much as the instruction count.
+// The CTA is warp-specialised and software-pipelined over the chunks of all chains it owns (27 warps):
+//   warp 0       TMA producer: K/Q tiles two chunks ahead (3 slots), V one chunk ahead (1 slot)
+//   warp 1       issues the chain MMAs (U^T, S0 W^T, S0 Q^T, Dl^T P^T, state update)
+//   warp 2       issues the Gram MMAs, two chunks ahead of the chain
+//   warp 3       decay warp: loads g and beta up to three chunks ahead, scans the log-decay and publishes the
+//                per-chunk decay factors
+//   warps 4-11   group G1 (two warps per TMEM lane window): Gram post-processing (A, P) of chunk k+1, then
+//                T', T'' of chunk k once its inverse is ready, and the W^T epilogue of chunk k-1
+//   warps 12-19  chain group: Delta epilogue, state conversion and pre-scaling, final state (chunk j)
+//   warps 20-21  group G2: the triangular solve of chunk k, overlapped with G1's other work
+//   warp 22      issues the W^T MMAs
+//   warps 23-26  output group: output epilogue of chunk j, off the chain's critical path
+// Every per-chunk loop is kept rolled with 16-column TMEM accesses: straight-line code larger than the
+// instruction caches runs at a fraction of the issue rate, so the static footprint matters as much as the
+// instruction count.
 // Chains (request, v-head) are ordered longest-first by the scheduler kernel and dealt to CTAs in
 // snake order, so each role can walk its CTA's chunk sequence without any broadcast.  Padding rows
 // of a ragged last chunk get g = 0 and beta = 0, which makes them inert; their outputs are not stored.
@@ -43,7 +47,7 @@ using namespace ptx;
 constexpr int LDA = 72;                       // bf16 row stride of the A and X scratch (144 B: conflict-free ldmatrix)
 constexpr int LDM = 40;                       // bf16 row stride of the merge scratch (80 B)
 constexpr float kLog2e = 1.4426950408889634f;
-constexpr int kThreads = 640;      // 3 single-lane role warps (+1 idle), 8 pre warps, 8 chain warps
+constexpr int kThreads = 864;      // 27 warps, see the role table above
 constexpr int kWgThreads = 256;
 
 // ---- shared memory map (bytes from a 1024-aligned base) ---------------------------------------
@@ -54,9 +58,9 @@ constexpr uint32_t SM_WT = 114688;            // W^T [dk][t] bf16, 128 rows x 12
 constexpr uint32_t SM_TP = 131072;            // 2 x T'  [t][s] bf16                                        16 KB
 constexpr uint32_t SM_TPP = 147456;           // T'' [t][s] bf16                                             8 KB
 constexpr uint32_t SM_P = 155648;             // 3 x P [t][s] bf16                                          24 KB
-constexpr uint32_t SM_OST = 180224;           // O staging [t][dv] bf16                                     16 KB
-constexpr uint32_t SM_AH = 196608;            // A bf16 [64][LDA]
-constexpr uint32_t SM_XH = SM_AH + 64 * LDA * 2;   // X = (I + A)^-1 bf16 [64][LDA]
+constexpr uint32_t SM_AH = 180224;            // 2 x A bf16 [64][LDA]
+constexpr uint32_t AH_BYTES = 64 * LDA * 2;
+constexpr uint32_t SM_XH = SM_AH + 2 * AH_BYTES;   // X = (I + A)^-1 bf16 [64][LDA]
 constexpr uint32_t SM_MH = SM_XH + 64 * LDA * 2;   // merge scratch bf16 [32][LDM]
 constexpr uint32_t SM_MISC = ((SM_MH + 32 * LDM * 2 + 1023) / 1024) * 1024;
 
@@ -66,7 +70,8 @@ enum Bar {
     B_GRAM_READ, B_WACC_READ, B_TPP_READY,
     B_PRE_DONE0, B_PRE_DONE1, B_D_READY, B_SBF_READY, B_ACC23_FREE,
     B_DECAY_READY0, B_DECAY_READY1, B_DECAY_READY2, B_DECAY_READY3,
-    B_DECAY_FREE0, B_DECAY_FREE1, B_DECAY_FREE2, B_DECAY_FREE3, NUM_BARS
+    B_DECAY_FREE0, B_DECAY_FREE1, B_DECAY_FREE2, B_DECAY_FREE3,
+    B_A_READY0, B_A_READY1, B_A_FREE0, B_A_FREE1, B_X_READY, B_X_FREE, NUM_BARS
 };
 
 // G2 = log2(e) * cumulative log-decay; bE = beta e^G; eG = e^G; eRest = e^{G_C - G}
@@ -202,9 +207,14 @@ struct Ctx {
     {
         const uint32_t b = bar(i);
         if (mbar_try_wait(b, parity)) return true;
+        return wait_slow(b, parity, misc);
+    }
+    // kept out of line: the kernel has some sixty wait sites and its static code size matters
+    __device__ __noinline__ static bool wait_slow(uint32_t b, uint32_t parity, Misc* misc)
+    {
         if (misc->abort) return true;
         const uint64_t t0 = globaltimer_ns();
-        for (uint32_t it = 0;; ++it) {
+        for (;;) {
             // suspended in hardware until the phase completes (or ~20 us pass): no polling instructions
             if (mbar_try_wait_hint(b, parity, 20000u)) return true;
             if (misc->abort) return true;
@@ -330,14 +340,14 @@ __device__ void role_producer(const Ctx& cx, const TcParams& prm, const CUtensor
 __device__ __forceinline__ uint64_t desc_add(uint64_t d, uint32_t bytes) { return d + (uint64_t)(bytes >> 4); }
 
 // ================================================================================================
-// warp 2: intra-chunk MMAs (Gram and W^T) for the chunk the pre group works on
+// warp 2: Gram MMAs.  Gram(j) needs the K/Q tiles of chunk j and the accumulator read by chunk j-1.
 // ================================================================================================
-__device__ void role_mma_pre(const Ctx& cx, const TcParams& prm)
+__device__ void role_mma_gram(const Ctx& cx, const TcParams& prm)
 {
-    ChunkCursor cg;                       // cursor of the Gram MMAs, one chunk ahead of the W^T MMAs
-    cg.init(&prm.p, prm.s.order);
-    const uint64_t d_tpp = smem_desc_sw128(cx.sb + SM_TPP, 16, 1024);
-    auto gram = [&](uint32_t j) {         // Gram(j): needs the K/Q tiles and the accumulator read by chunk j-1
+    ChunkCursor cc;
+    cc.init(&prm.p, prm.s.order);
+#pragma unroll 1
+    for (uint32_t j = 0; cc.valid; ++j, cc.advance()) {
         const uint32_t slot = j % 3u;
         const uint64_t d_kq = smem_desc_sw128(cx.sb + SM_KQ + slot * KQ_SLOT, 16, 1024);   // [K;Q] rows, K-major
         cx.wait(B_FULL_KQ0 + slot, (j / 3u) & 1u);
@@ -352,8 +362,19 @@ __device__ void role_mma_pre(const Ctx& cx, const TcParams& prm)
             mma_commit(cx.bar(B_GRAM_DONE));
         }
         __syncwarp();
-    };
-    auto wmma = [&](uint32_t j) {         // W^T(j) = K^T T''^T: needs T''(j) and the accumulator read by chunk j-1
+    }
+}
+
+// ================================================================================================
+// warp 22: W^T MMAs.  W^T(j) = K^T T''^T needs T''(j) and the accumulator read by chunk j-1.
+// ================================================================================================
+__device__ void role_mma_w(const Ctx& cx, const TcParams& prm)
+{
+    ChunkCursor cc;
+    cc.init(&prm.p, prm.s.order);
+    const uint64_t d_tpp = smem_desc_sw128(cx.sb + SM_TPP, 16, 1024);
+#pragma unroll 1
+    for (uint32_t j = 0; cc.valid; ++j, cc.advance()) {
         const uint64_t d_kt = smem_desc_sw128(cx.sb + SM_KQ + (j % 3u) * KQ_SLOT, 16384, 1024);   // K^T, M-major
         cx.wait(B_TPP_READY, j & 1u);
         if (j >= 1) cx.wait(B_WACC_READ, (j - 1) & 1u);
@@ -365,19 +386,7 @@ __device__ void role_mma_pre(const Ctx& cx, const TcParams& prm)
             mma_commit(cx.bar(B_W_DONE));
         }
         __syncwarp();
-    };
-    if (!cg.valid) return;
-    gram(0);
-    cg.advance();
-    uint32_t j = 0;
-#pragma unroll 1
-    for (;; ++j) {
-        if (j >= 1) wmma(j - 1);
-        if (!cg.valid) break;
-        gram(j + 1);
-        cg.advance();
     }
-    wmma(j);
 }
 
 // ================================================================================================
@@ -490,35 +499,158 @@ __device__ void role_decay(const Ctx& cx, const TcParams& prm)
     }
 }
 
-// ================================================================================================
-// warps 4-11: pre group (intra-chunk stage of the chunk one ahead of the chain)
-// ================================================================================================
-__device__ void role_pre(const Ctx& cx, const TcParams& prm, int wtid)
+// Number of 64-row chunks this CTA processes over all of its chains.
+__device__ __noinline__ uint32_t count_chunks(const TcParams& prm)
 {
-    const Problem& p = prm.p;
+    ChunkCursor cc;
+    cc.init(&prm.p, prm.s.order);
+    uint32_t n = 0;
+    while (cc.valid) { n += (uint32_t)cc.nchunks; cc.next_chain(); }
+    return n;
+}
+
+// ================================================================================================
+// warps 4-11: group G1.  Per iteration k: W^T epilogue of chunk k-1, Gram post-processing of chunk k+1
+// (writes A for the solve and the operand P), then T' and T'' of chunk k once group G2 has inverted it.
+// ================================================================================================
+__device__ void role_g1(const Ctx& cx, const TcParams& prm, int wtid)
+{
     const int lane = wtid & 31, pw = wtid >> 5;          // pw = 0..7
     const int w4 = pw & 3, hf = pw >> 2;                 // TMEM lane window, column half
     const uint32_t tl = cx.tmem + ((uint32_t)(w4 * 32) << 16);
-    uint8_t* AH = cx.sm + SM_AH;
     uint8_t* XH = cx.sm + SM_XH;
-    uint8_t* MH = cx.sm + SM_MH;
-    const uint32_t ah = cx.sb + SM_AH, xh = cx.sb + SM_XH, mh = cx.sb + SM_MH;
     Misc* misc = cx.misc;
-    ChunkCursor cc;
-    cc.init(&p, prm.s.order);
+    const uint32_t J = count_chunks(prm);
     GDN_TIMERS(long long tt_[16] = {0}; long long tl_ = clock64(); int nch = 0;)
-    // W^T epilogue of chunk jw (warps 4-7, all 64 columns of their lane window): bf16 rows [dk][t] as the
-    // N-major operand of the S0 W^T MMA; completes the operand set of chunk jw
-    auto w_epilogue = [&](uint32_t jw) {
-        cx.wait(B_W_DONE, jw & 1u);
+
+    // ---- Gram tile of chunk c -> A (bf16 scratch for the solve) and P (bf16 operand), 16 columns at a time
+    auto post = [&](uint32_t c) {
+        const Decay& dc = misc->decay[c & 3u];
+        cx.wait(B_DECAY_READY0 + (c & 3u), (c >> 2) & 1u);       // decay factors of this chunk are published
+        // this thread's row of the Gram tile: lane windows 0,1 hold K K^T rows, 2,3 hold Q K^T rows
+        const int t = ((w4 & 1) << 5) + lane;
+        const bool isA = w4 < 2;
+        const float G2t = dc.G2[t];
+        const float rowscale = isA ? dc.beta[t] : 1.f;
+        const int t_lim = isA ? t : t + 1;                      // keep columns s < t_lim
+        cx.wait(B_GRAM_DONE, c & 1u);
         tc_fence_after();
-        // W^T is single-buffered: the S0 W^T MMA of chunk jw-1 must have read it
-        if (jw >= 1) cx.wait(B_MMA1_DONE, (jw - 1) & 1u);
-        const int drow = w4 * 32 + lane;                      // dk index = TMEM lane
+        // buffers: P of chunk c was last read by the MMAs of chunk c-3, A by the solve of chunk c-2
+        if (c >= 3) cx.wait(B_P_FREE0 + c % 3u, ((c / 3u) - 1u) & 1u);
+        if (c >= 2) cx.wait(B_A_FREE0 + (c & 1u), ((c >> 1) - 1u) & 1u);
+        uint8_t* AH = cx.sm + SM_AH + (c & 1u) * AH_BYTES;
+        uint8_t* prow = cx.sm + SM_P + (c % 3u) * 8192 + t * 128;
+        // column blocks are dealt so that each warp of a lane window gets one block that touches the
+        // diagonal and one that does not: half 0 -> blocks {0, 2}, half 1 -> blocks {1, 3}
+        const bool lower_rows = (w4 & 1) != 0;                  // rows 32-63
+        const float rowf = lower_rows ? ex2_approx(G2t - dc.G2mid) * rowscale : 0.f;
+#pragma unroll 1
+        for (int g = 0; g < 2; ++g) {
+            const int cb = hf + 2 * g, c0 = 16 * cb;
+            if (c0 > ((w4 & 1) << 5) + 31) {                    // block entirely above the diagonal (warp-uniform)
+                if (!isA) {
+                    *reinterpret_cast<uint4*>(prow + (((2 * cb) ^ (t & 7)) << 4)) = make_uint4(0u, 0u, 0u, 0u);
+                    *reinterpret_cast<uint4*>(prow + (((2 * cb + 1) ^ (t & 7)) << 4)) = make_uint4(0u, 0u, 0u, 0u);
+                }
+                continue;
+            }
+            uint32_t acc[16];
+            tmem_ld16(tl + TM_GRAM + c0, acc);
+            tmem_ld_wait();
+            float vals[16];
+            if (lower_rows && cb < 2) {
+                // every column precedes every row of this warp: Gam = rowf * colf, no mask, no exp
+#pragma unroll
+                for (int i4 = 0; i4 < 4; ++i4) {
+                    const float4 cf = *reinterpret_cast<const float4*>(&dc.colf[c0 + 4 * i4]);
+                    vals[4 * i4 + 0] = (rowf * cf.x) * __uint_as_float(acc[4 * i4 + 0]);
+                    vals[4 * i4 + 1] = (rowf * cf.y) * __uint_as_float(acc[4 * i4 + 1]);
+                    vals[4 * i4 + 2] = (rowf * cf.z) * __uint_as_float(acc[4 * i4 + 2]);
+                    vals[4 * i4 + 3] = (rowf * cf.w) * __uint_as_float(acc[4 * i4 + 3]);
+                }
+            } else {
+#pragma unroll
+                for (int i4 = 0; i4 < 4; ++i4) {
+                    const float4 gs = *reinterpret_cast<const float4*>(&dc.G2[c0 + 4 * i4]);
+                    const float gss[4] = {gs.x, gs.y, gs.z, gs.w};
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        const int i = 4 * i4 + e;
+                        // masked entries may overflow to inf / NaN before the select discards them
+                        const float f = ex2_approx(G2t - gss[e]) * rowscale;
+                        vals[i] = (c0 + i < t_lim) ? f * __uint_as_float(acc[i]) : 0.f;
+                    }
+                }
+            }
+            uint4 u[2];
+#pragma unroll
+            for (int c8 = 0; c8 < 2; ++c8) {
+                u[c8].x = pack_bf16x2(vals[c8 * 8 + 0], vals[c8 * 8 + 1]);
+                u[c8].y = pack_bf16x2(vals[c8 * 8 + 2], vals[c8 * 8 + 3]);
+                u[c8].z = pack_bf16x2(vals[c8 * 8 + 4], vals[c8 * 8 + 5]);
+                u[c8].w = pack_bf16x2(vals[c8 * 8 + 6], vals[c8 * 8 + 7]);
+            }
+            if (isA) {
+                uint8_t* arow = AH + (t * LDA + c0) * 2;
+                *reinterpret_cast<uint4*>(arow) = u[0];
+                *reinterpret_cast<uint4*>(arow + 16) = u[1];
+            } else {
+                *reinterpret_cast<uint4*>(prow + (((2 * cb) ^ (t & 7)) << 4)) = u[0];
+                *reinterpret_cast<uint4*>(prow + (((2 * cb + 1) ^ (t & 7)) << 4)) = u[1];
+            }
+        }
+        tc_fence_before();
+        warp_arrive(cx.bar(B_GRAM_READ), lane);                 // the accumulator may take the next Gram tile
+        fence_proxy_async_smem();                               // P is an MMA operand
+        warp_arrive(cx.bar(B_A_READY0 + (c & 1u)), lane);       // A of chunk c is complete: the solve may start
+    };
+
+    // ---- T'' = X diag(beta e^G) (operand of the W^T MMA), T' = X diag(beta) (operand of the U^T MMA) ------
+    auto t_write = [&](uint32_t k) {
+        const Decay& dc = misc->decay[k & 3u];
+        cx.wait(B_X_READY, k & 1u);
+        // the T' buffer of chunk k was last read by the U^T MMA of chunk k-2; T'' by the W^T MMA of chunk k-1,
+        // whose completion the W^T epilogue of this iteration has already waited for
+        if (k >= 2) cx.wait(B_TP_FREE0 + (k & 1u), ((k >> 1) - 1u) & 1u);
+        const int tt = wtid >> 2, q = wtid & 3, c0 = 16 * q;   // row, 16-column quarter
+        uint32_t w1[8], w2[8];
+#pragma unroll
+        for (int c8 = 0; c8 < 2; ++c8) {
+            const uint4 xv = *reinterpret_cast<const uint4*>(XH + (tt * LDA + c0 + 8 * c8) * 2);
+            const uint32_t xw[4] = {xv.x, xv.y, xv.z, xv.w};
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const int s0 = c0 + 8 * c8 + 2 * e;
+                const float2 bv = *reinterpret_cast<const float2*>(&dc.beta[s0]);
+                const float2 ev = *reinterpret_cast<const float2*>(&dc.bE[s0]);
+                const float x0 = (s0 <= tt) ? bf_lo(xw[e]) : 0.f, x1 = (s0 + 1 <= tt) ? bf_hi(xw[e]) : 0.f;
+                w1[4 * c8 + e] = pack_bf16x2(x0 * bv.x, x1 * bv.y);
+                w2[4 * c8 + e] = pack_bf16x2(x0 * ev.x, x1 * ev.y);
+            }
+        }
+        warp_arrive(cx.bar(B_X_FREE), lane);                    // X has been read: the next solve may overwrite it
+        const uint32_t o0 = tt * 128 + (((2 * q) ^ (tt & 7)) << 4), o1 = tt * 128 + (((2 * q + 1) ^ (tt & 7)) << 4);
+        uint8_t* tp = cx.sm + SM_TP + (k & 1u) * 8192;
+        *reinterpret_cast<uint4*>(tp + o0) = make_uint4(w1[0], w1[1], w1[2], w1[3]);
+        *reinterpret_cast<uint4*>(tp + o1) = make_uint4(w1[4], w1[5], w1[6], w1[7]);
+        *reinterpret_cast<uint4*>(cx.sm + SM_TPP + o0) = make_uint4(w2[0], w2[1], w2[2], w2[3]);
+        *reinterpret_cast<uint4*>(cx.sm + SM_TPP + o1) = make_uint4(w2[4], w2[5], w2[6], w2[7]);
+        fence_proxy_async_smem();
+        warp_arrive(cx.bar(B_TPP_READY), lane);
+    };
+
+    // ---- W^T epilogue of chunk c: bf16 rows [dk][t] as the N-major operand of the S0 W^T MMA; completes the
+    // operand set of chunk c (each warp converts 32 columns of its lane window)
+    auto w_epilogue = [&](uint32_t c) {
+        cx.wait(B_W_DONE, c & 1u);
+        tc_fence_after();
+        // W^T is single-buffered: the S0 W^T MMA of chunk c-1 must have read it
+        if (c >= 1) cx.wait(B_MMA1_DONE, (c - 1) & 1u);
+        const int drow = w4 * 32 + lane;                        // dk index = TMEM lane
         uint8_t* wrow = cx.sm + SM_WT + drow * 128;
 #pragma unroll 1
-        for (int g = 0; g < 4; ++g) {
-            const int c0 = 16 * g;
+        for (int g = 0; g < 2; ++g) {
+            const int c0 = 32 * hf + 16 * g;
             uint32_t acc[16];
             tmem_ld16(tl + TM_WACC + c0, acc);
             tmem_ld_wait();
@@ -533,174 +665,106 @@ __device__ void role_pre(const Ctx& cx, const TcParams& prm, int wtid)
             }
         }
         tc_fence_before();
-        warp_arrive(cx.bar(B_WACC_READ), lane);            // the accumulator may take the next W^T tile
+        warp_arrive(cx.bar(B_WACC_READ), lane);                 // the accumulator may take the next W^T tile
         fence_proxy_async_smem();
-        warp_arrive(cx.bar(B_PRE_DONE0 + (jw & 1u)), lane);
+        warp_arrive(cx.bar(B_PRE_DONE0 + (c & 1u)), lane);
     };
-    auto solve_sync = [&]() { asm volatile("bar.sync 3, 128;" ::: "memory"); };
-    uint32_t j_total = 0;
+
+    if (J == 0) return;
+    post(0);
 #pragma unroll 1
-    for (uint32_t j = 0; cc.valid; ++j, cc.advance()) {
-        j_total = j + 1;
-        Decay& dc = misc->decay[j & 3u];
-        GDN_DBG(const bool dbg = prm.debug && blockIdx.x == 0 && cc.r == 0 && cc.c < 2;
-                float* dbase = prm.debug + cc.c * DBG_STRIDE;)
-        cx.wait(B_DECAY_READY0 + (j & 3u), (j >> 2) & 1u);     // decay factors of this chunk are published
-        // this thread's row of the Gram tile: lane windows 0,1 hold K K^T rows, 2,3 hold Q K^T rows
-        const int t = ((w4 & 1) << 5) + lane;
-        const bool isA = w4 < 2;
-        const float G2t = dc.G2[t];
-        const float rowscale = isA ? dc.beta[t] : 1.f;
-        const int t_lim = isA ? t : t + 1;               // keep columns s < t_lim
+    for (uint32_t k = 0; k < J; ++k) {
+        if (k >= 1) w_epilogue(k - 1);       // first: it completes the operand set the chain is waiting for
         GDN_T(0);
-
-        // ---- Gram tile -> A (fp32 scratch) and P (bf16 operand), 16 columns at a time ----------------------
-        cx.wait(B_GRAM_DONE, j & 1u);
+        if (k + 1 < J) post(k + 1);          // overlaps the solve of chunk k
         GDN_T(1);
-        tc_fence_after();
-        // the P buffer of chunk j was last read by the MMAs of chunk j-3
-        if (j >= 3) cx.wait(B_P_FREE0 + j % 3u, ((j / 3u) - 1u) & 1u);
-        {
-            uint8_t* prow = cx.sm + SM_P + (j % 3u) * 8192 + t * 128;
-            // column blocks are dealt so that each warp of a lane window gets one block that touches the
-            // diagonal and one that does not: half 0 -> blocks {0, 2}, half 1 -> blocks {1, 3}
-            const bool lower_rows = (w4 & 1) != 0;             // rows 32-63
-            const float rowf = lower_rows ? ex2_approx(G2t - dc.G2mid) * rowscale : 0.f;
-#pragma unroll 1
-            for (int g = 0; g < 2; ++g) {
-                const int cb = hf + 2 * g, c0 = 16 * cb;
-                if (c0 > ((w4 & 1) << 5) + 31) {          // block entirely above the diagonal (warp-uniform)
-                    if (!isA) {
-                        *reinterpret_cast<uint4*>(prow + (((2 * cb) ^ (t & 7)) << 4)) = make_uint4(0u, 0u, 0u, 0u);
-                        *reinterpret_cast<uint4*>(prow + (((2 * cb + 1) ^ (t & 7)) << 4)) = make_uint4(0u, 0u, 0u, 0u);
-                    }
-                    continue;
-                }
-                uint32_t acc[16];
-                tmem_ld16(tl + TM_GRAM + c0, acc);
-                tmem_ld_wait();
-#ifdef GDN_TC_DEBUG
-                if (dbg) {
-#pragma unroll
-                    for (int i = 0; i < 16; ++i) dbase[(w4 * 32 + lane) * 64 + c0 + i] = __uint_as_float(acc[i]);
-                }
-#endif
-                float vals[16];
-                if (lower_rows && cb < 2) {
-                    // every column precedes every row of this warp: Gam = rowf * colf, no mask, no exp
-#pragma unroll
-                    for (int i4 = 0; i4 < 4; ++i4) {
-                        const float4 cf = *reinterpret_cast<const float4*>(&dc.colf[c0 + 4 * i4]);
-                        vals[4 * i4 + 0] = (rowf * cf.x) * __uint_as_float(acc[4 * i4 + 0]);
-                        vals[4 * i4 + 1] = (rowf * cf.y) * __uint_as_float(acc[4 * i4 + 1]);
-                        vals[4 * i4 + 2] = (rowf * cf.z) * __uint_as_float(acc[4 * i4 + 2]);
-                        vals[4 * i4 + 3] = (rowf * cf.w) * __uint_as_float(acc[4 * i4 + 3]);
-                    }
-                } else {
-#pragma unroll
-                    for (int i4 = 0; i4 < 4; ++i4) {
-                        const float4 gs = *reinterpret_cast<const float4*>(&dc.G2[c0 + 4 * i4]);
-                        const float gss[4] = {gs.x, gs.y, gs.z, gs.w};
-#pragma unroll
-                        for (int e = 0; e < 4; ++e) {
-                            const int i = 4 * i4 + e;
-                            // masked entries may overflow to inf / NaN before the select discards them
-                            const float f = ex2_approx(G2t - gss[e]) * rowscale;
-                            vals[i] = (c0 + i < t_lim) ? f * __uint_as_float(acc[i]) : 0.f;
-                        }
-                    }
-                }
-                if (isA) {
-                    uint8_t* arow = AH + (t * LDA + c0) * 2;
-#pragma unroll
-                    for (int c8 = 0; c8 < 2; ++c8) {
-                        uint4 u;
-                        u.x = pack_bf16x2(vals[c8 * 8 + 0], vals[c8 * 8 + 1]);
-                        u.y = pack_bf16x2(vals[c8 * 8 + 2], vals[c8 * 8 + 3]);
-                        u.z = pack_bf16x2(vals[c8 * 8 + 4], vals[c8 * 8 + 5]);
-                        u.w = pack_bf16x2(vals[c8 * 8 + 6], vals[c8 * 8 + 7]);
-                        *reinterpret_cast<uint4*>(arow + c8 * 16) = u;
-                    }
-                } else {
-#pragma unroll
-                    for (int c8 = 0; c8 < 2; ++c8) {
-                        uint4 u;
-                        u.x = pack_bf16x2(vals[c8 * 8 + 0], vals[c8 * 8 + 1]);
-                        u.y = pack_bf16x2(vals[c8 * 8 + 2], vals[c8 * 8 + 3]);
-                        u.z = pack_bf16x2(vals[c8 * 8 + 4], vals[c8 * 8 + 5]);
-                        u.w = pack_bf16x2(vals[c8 * 8 + 6], vals[c8 * 8 + 7]);
-                        *reinterpret_cast<uint4*>(prow + (((2 * cb + c8) ^ (t & 7)) << 4)) = u;
-                    }
-                }
-            }
-        }
-        tc_fence_before();
-        warp_arrive(cx.bar(B_GRAM_READ), lane);            // the accumulator may take the next Gram tile
-        wg_sync(1);
+        t_write(k);
         GDN_T(2);
+        GDN_TIMERS(++nch;)
+    }
+    w_epilogue(J - 1);
+#ifdef GDN_TC_PROFILE
+    if (prm.debug && blockIdx.x == 0 && wtid == 0 && nch > 0) {
+        float* d = prm.debug + 5 * 48;
+        d[0] = (float)nch;
+        for (int i = 0; i < 12; ++i) d[1 + i] = (float)tt_[i] / nch;
+    }
+#endif
+}
 
-        // ---- X = (I + A)^-1 ----------------------------------------------------------------------------
-        // warps 0 and 1 each invert one 32 x 32 diagonal half without any cross-warp barrier:
-        //   level 0  : its four 8 x 8 diagonal blocks by forward substitution in fp32
-        //   level 0.5: 8 -> 16 merges, level 1: the 16 -> 32 merge X[hi][lo] = -X[hi][hi] (A[hi][lo] X[lo][lo]),
-        //              both on mma.sync with ldmatrix-fed bf16 fragments
-        if (pw >= 4) {
-            // warps 4-7 (one per TMEM lane window) are not needed by the solve: they convert W^T of the
-            // previous chunk meanwhile
-            if (j >= 1) w_epilogue(j - 1);
+// ================================================================================================
+// warps 20-21: group G2, X = (I + A)^-1 of chunk k while G1 works on its neighbours.  Each warp inverts one
+// 32 x 32 diagonal half without any cross-warp barrier:
+//   level 0  : its four 8 x 8 diagonal blocks by forward substitution in fp32
+//   level 0.5: 8 -> 16 merges, level 1: the 16 -> 32 merge X[hi][lo] = -X[hi][hi] (A[hi][lo] X[lo][lo]),
+//   level 2  : X[32:64][0:32] = -X22 (A21 X11), two 16 x 16 tiles per warp,
+// the merges on mma.sync with ldmatrix-fed bf16 fragments.
+// ================================================================================================
+__device__ void role_g2(const Ctx& cx, const TcParams& prm, int wtid)
+{
+    const int lane = wtid & 31, pw = wtid >> 5;          // pw = 0, 1
+    uint8_t* XH = cx.sm + SM_XH;
+    uint8_t* MH = cx.sm + SM_MH;
+    const uint32_t xh = cx.sb + SM_XH, mh = cx.sb + SM_MH;
+    const uint32_t J = count_chunks(prm);
+    auto pair_sync = [&]() { asm volatile("bar.sync 3, 64;" ::: "memory"); };
+    GDN_TIMERS(long long tt_[16] = {0}; long long tl_ = clock64(); int nch = 0;)
+#pragma unroll 1
+    for (uint32_t k = 0; k < J; ++k) {
+        const uint8_t* AH = cx.sm + SM_AH + (k & 1u) * AH_BYTES;
+        const uint32_t ah = cx.sb + SM_AH + (k & 1u) * AH_BYTES;
+        cx.wait(B_A_READY0 + (k & 1u), (k >> 1) & 1u);
+        if (k >= 1) cx.wait(B_X_FREE, (k - 1) & 1u);           // T', T'' of chunk k-1 have been formed from X
+        GDN_T(0);
+        {
+            const int bb = 4 * pw + (lane >> 3), b = 8 * bb, jj = lane & 7;
+            float x[8];
+#pragma unroll
+            for (int r = 0; r < 8; ++r) x[r] = (r == jj) ? 1.f : 0.f;
+#pragma unroll
+            for (int r = 1; r < 8; ++r) {
+                const uint4 a4 = *reinterpret_cast<const uint4*>(AH + ((b + r) * LDA + b) * 2);
+                const uint32_t wds[4] = {a4.x, a4.y, a4.z, a4.w};
+                float acc0 = 0.f, acc1 = 0.f;
+#pragma unroll
+                for (int s2 = 0; s2 < r; ++s2) {
+                    const float a = (s2 & 1) ? bf_hi(wds[s2 >> 1]) : bf_lo(wds[s2 >> 1]);
+                    if (s2 & 1) acc1 = fmaf(a, x[s2], acc1); else acc0 = fmaf(a, x[s2], acc0);
+                }
+                x[r] = (r > jj) ? -(acc0 + acc1) : x[r];
+            }
+            const int zc = b + 8;                              // upper-right 8 x 8 of the 16 x 16 parent block
+#pragma unroll
+            for (int r = 0; r < 8; ++r) {
+                *reinterpret_cast<__nv_bfloat16*>(XH + ((b + r) * LDA + b + jj) * 2) = __float2bfloat16_rn(x[r]);
+                if (!(bb & 1)) *reinterpret_cast<uint16_t*>(XH + ((b + r) * LDA + zc + jj) * 2) = 0;
+            }
         }
-        if (pw < 2) {
-            // level 0: four 8 x 8 diagonal blocks per warp (lane & 7 owns a column of block 4 pw + lane / 8)
-            {
-                const int bb = 4 * pw + (lane >> 3), b = 8 * bb, jj = lane & 7;
-                float x[8];
-#pragma unroll
-                for (int r = 0; r < 8; ++r) x[r] = (r == jj) ? 1.f : 0.f;
-#pragma unroll
-                for (int r = 1; r < 8; ++r) {
-                    const uint4 a4 = *reinterpret_cast<const uint4*>(AH + ((b + r) * LDA + b) * 2);
-                    const uint32_t wds[4] = {a4.x, a4.y, a4.z, a4.w};
-                    float acc0 = 0.f, acc1 = 0.f;
-#pragma unroll
-                    for (int s2 = 0; s2 < r; ++s2) {
-                        const float a = (s2 & 1) ? bf_hi(wds[s2 >> 1]) : bf_lo(wds[s2 >> 1]);
-                        if (s2 & 1) acc1 = fmaf(a, x[s2], acc1); else acc0 = fmaf(a, x[s2], acc0);
-                    }
-                    x[r] = (r > jj) ? -(acc0 + acc1) : x[r];
-                }
-                const int zc = (bb & 1) ? b - 8 : b + 8;      // the other 8 columns of this block's 16 x 16 parent
-#pragma unroll
-                for (int r = 0; r < 8; ++r) {
-                    *reinterpret_cast<__nv_bfloat16*>(XH + ((b + r) * LDA + b + jj) * 2) = __float2bfloat16_rn(x[r]);
-                    if (!(bb & 1)) *reinterpret_cast<uint16_t*>(XH + ((b + r) * LDA + zc + jj) * 2) = 0;   // upper-right 8 x 8
-                }
-            }
+        __syncwarp();
+        {
+            const int i = (lane >> 3) & 1, rr = lane & 7, b16 = 32 * pw + 16 * i;
+            const int g = lane >> 2, t4 = lane & 3;
+            uint32_t a[2], bx[2];
+            ldm_x2(a, ah + ((b16 + 8 + rr) * LDA + b16) * 2);                    // A21 of both blocks
+            ldm_x2_trans(bx, xh + ((b16 + rr) * LDA + b16) * 2);                  // X11 of both blocks
+            float m0[4] = {0.f, 0.f, 0.f, 0.f}, m1[4] = {0.f, 0.f, 0.f, 0.f};
+            mma_8x8(m0, a[0], bx[0]);
+            mma_8x8(m1, a[1], bx[1]);
+            *reinterpret_cast<uint32_t*>(MH + ((16 * pw + g) * LDM + 2 * t4) * 2) = pack_bf16x2(m0[0], m0[1]);
+            *reinterpret_cast<uint32_t*>(MH + ((16 * pw + 8 + g) * LDM + 2 * t4) * 2) = pack_bf16x2(m1[0], m1[1]);
             __syncwarp();
-            // level 0.5: inside each of this warp's two 16 x 16 blocks, X21 = -X22 (A21 X11) with 8 x 8 pieces
-            {
-                const int i = (lane >> 3) & 1, rr = lane & 7, b16 = 32 * pw + 16 * i;
-                const int g = lane >> 2, t4 = lane & 3;
-                uint32_t a[2], bx[2];
-                ldm_x2(a, ah + ((b16 + 8 + rr) * LDA + b16) * 2);                    // A21 of both blocks
-                ldm_x2_trans(bx, xh + ((b16 + rr) * LDA + b16) * 2);                  // X11 of both blocks
-                float m0[4] = {0.f, 0.f, 0.f, 0.f}, m1[4] = {0.f, 0.f, 0.f, 0.f};
-                mma_8x8(m0, a[0], bx[0]);
-                mma_8x8(m1, a[1], bx[1]);
-                // M_i at rows 16 pw + 8 i of the merge scratch, columns 0-7
-                *reinterpret_cast<uint32_t*>(MH + ((16 * pw + g) * LDM + 2 * t4) * 2) = pack_bf16x2(m0[0], m0[1]);
-                *reinterpret_cast<uint32_t*>(MH + ((16 * pw + 8 + g) * LDM + 2 * t4) * 2) = pack_bf16x2(m1[0], m1[1]);
-                __syncwarp();
-                uint32_t a2[2], bm[2];
-                ldm_x2(a2, xh + ((b16 + 8 + rr) * LDA + b16 + 8) * 2);               // X22 of both blocks
-                ldm_x2_trans(bm, mh + ((16 * pw + 8 * i + rr) * LDM) * 2);           // M of both blocks
-                float d0[4] = {0.f, 0.f, 0.f, 0.f}, d1[4] = {0.f, 0.f, 0.f, 0.f};
-                mma_8x8(d0, a2[0], bm[0]);
-                mma_8x8(d1, a2[1], bm[1]);
-                const int c0b = 32 * pw, c1b = 32 * pw + 16;
-                *reinterpret_cast<uint32_t*>(XH + ((c0b + 8 + g) * LDA + c0b + 2 * t4) * 2) = pack_bf16x2(-d0[0], -d0[1]);
-                *reinterpret_cast<uint32_t*>(XH + ((c1b + 8 + g) * LDA + c1b + 2 * t4) * 2) = pack_bf16x2(-d1[0], -d1[1]);
-            }
-            __syncwarp();
+            uint32_t a2[2], bm[2];
+            ldm_x2(a2, xh + ((b16 + 8 + rr) * LDA + b16 + 8) * 2);               // X22 of both blocks
+            ldm_x2_trans(bm, mh + ((16 * pw + 8 * i + rr) * LDM) * 2);           // M of both blocks
+            float d0[4] = {0.f, 0.f, 0.f, 0.f}, d1[4] = {0.f, 0.f, 0.f, 0.f};
+            mma_8x8(d0, a2[0], bm[0]);
+            mma_8x8(d1, a2[1], bm[1]);
+            const int c0b = 32 * pw, c1b = 32 * pw + 16;
+            *reinterpret_cast<uint32_t*>(XH + ((c0b + 8 + g) * LDA + c0b + 2 * t4) * 2) = pack_bf16x2(-d0[0], -d0[1]);
+            *reinterpret_cast<uint32_t*>(XH + ((c1b + 8 + g) * LDA + c1b + 2 * t4) * 2) = pack_bf16x2(-d1[0], -d1[1]);
+        }
+        __syncwarp();
+        {
             const int lo = 32 * pw, hi = 32 * pw + 16;
             float m[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
             tile16_mma(m, ah, LDA, hi, lo, xh, LDA, lo, lo, lane);               // A[hi][lo] X[lo][lo]
@@ -710,79 +774,37 @@ __device__ void role_pre(const Ctx& cx, const TcParams& prm, int wtid)
             tile16_mma(d, xh, LDA, hi, hi, mh, LDM, 16 * pw, 0, lane);           // X[hi][hi] M
             tile16_store(d, -1.f, XH, LDA, hi, lo, lane);
         }
-        if (pw < 4) solve_sync();
-        GDN_T(3);
-        // level 2: X[32:64][0:32] = -X22 (A21 X11); warps 0-3 take one 16 x 16 tile (mt, nt) each
+        pair_sync();
+        GDN_T(1);
+        // level 2: warp pw owns block row mt = pw of X[32:64][0:32], both block columns
         {
-            const int mt = (pw >> 1) & 1, nt = pw & 1;
-            if (pw < 4) {
+            const int mt = pw;
+#pragma unroll 1
+            for (int nt = 0; nt < 2; ++nt) {
                 float m[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
                 // X11 is lower triangular: block column nt starts at block row nt
                 for (int kb = nt; kb < 2; ++kb)
                     tile16_mma(m, ah, LDA, 32 + 16 * mt, 16 * kb, xh, LDA, 16 * kb, 16 * nt, lane);
                 tile16_store(m, 1.f, MH, LDM, 16 * mt, 16 * nt, lane);
-                solve_sync();
             }
-            if (pw < 4) {
+            warp_arrive(cx.bar(B_A_FREE0 + (k & 1u)), lane);   // last read of this chunk's A
+            pair_sync();
+#pragma unroll 1
+            for (int nt = 0; nt < 2; ++nt) {
                 float d[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
                 // X22 is lower triangular: block row mt ends at block column mt
                 for (int kb = 0; kb <= mt; ++kb)
                     tile16_mma(d, xh, LDA, 32 + 16 * mt, 32 + 16 * kb, mh, LDM, 16 * kb, 16 * nt, lane);
                 tile16_store(d, -1.f, XH, LDA, 32 + 16 * mt, 16 * nt, lane);
             }
-            wg_sync(1);
         }
-        GDN_T(4);
-#ifdef GDN_TC_DEBUG
-        if (dbg) for (int e = wtid; e < 4096; e += kWgThreads) dbase[8192 + e] = ((e & 63) <= (e >> 6)) ? __bfloat162float(*reinterpret_cast<const __nv_bfloat16*>(XH + ((e >> 6) * LDA + (e & 63)) * 2)) : 0.f;
-#endif
-        // ---- T'' = X diag(beta e^G) (operand of the W^T MMA), T' = X diag(beta) (operand of the U^T MMA) ----
-        // the T' buffer of chunk j was last read by the U^T MMA of chunk j-2
-        if (j >= 2) cx.wait(B_TP_FREE0 + (j & 1u), ((j >> 1) - 1u) & 1u);
-        GDN_T(9);
-        {
-            const int tt = wtid >> 2, q = wtid & 3, c0 = 16 * q;      // row, 16-column quarter
-            uint32_t w1[8], w2[8];
-#pragma unroll
-            for (int c8 = 0; c8 < 2; ++c8) {
-                const uint4 xv = *reinterpret_cast<const uint4*>(XH + (tt * LDA + c0 + 8 * c8) * 2);
-                const uint32_t xw[4] = {xv.x, xv.y, xv.z, xv.w};
-#pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    const int s0 = c0 + 8 * c8 + 2 * e;
-                    const float2 bv = *reinterpret_cast<const float2*>(&dc.beta[s0]);
-                    const float2 ev = *reinterpret_cast<const float2*>(&dc.bE[s0]);
-                    const float x0 = (s0 <= tt) ? bf_lo(xw[e]) : 0.f, x1 = (s0 + 1 <= tt) ? bf_hi(xw[e]) : 0.f;
-                    w1[4 * c8 + e] = pack_bf16x2(x0 * bv.x, x1 * bv.y);
-                    w2[4 * c8 + e] = pack_bf16x2(x0 * ev.x, x1 * ev.y);
-                }
-            }
-            const uint32_t o0 = tt * 128 + (((2 * q) ^ (tt & 7)) << 4), o1 = tt * 128 + (((2 * q + 1) ^ (tt & 7)) << 4);
-            uint8_t* tp = cx.sm + SM_TP + (j & 1u) * 8192;
-            *reinterpret_cast<uint4*>(tp + o0) = make_uint4(w1[0], w1[1], w1[2], w1[3]);
-            *reinterpret_cast<uint4*>(tp + o1) = make_uint4(w1[4], w1[5], w1[6], w1[7]);
-            *reinterpret_cast<uint4*>(cx.sm + SM_TPP + o0) = make_uint4(w2[0], w2[1], w2[2], w2[3]);
-            *reinterpret_cast<uint4*>(cx.sm + SM_TPP + o1) = make_uint4(w2[4], w2[5], w2[6], w2[7]);
-        }
-        GDN_T(10);
-        fence_proxy_async_smem();
-        GDN_T(11);
-        warp_arrive(cx.bar(B_TPP_READY), lane);
-        GDN_T(6);
-
-        GDN_T(8);
+        warp_arrive(cx.bar(B_X_READY), lane);
+        GDN_T(2);
         GDN_TIMERS(++nch;)
     }
-    if (pw >= 4 && j_total > 0) w_epilogue(j_total - 1);
-#ifdef GDN_TC_DEBUG
+#ifdef GDN_TC_PROFILE
     if (prm.debug && blockIdx.x == 0 && wtid == 0 && nch > 0) {
-        float* d = prm.debug + 2 * DBG_STRIDE;
-        d[0] = (float)nch;
-        for (int i = 0; i < 12; ++i) d[1 + i] = (float)tt_[i] / nch;
-    }
-#elif defined(GDN_TC_PROFILE)
-    if (prm.debug && blockIdx.x == 0 && wtid == 0 && nch > 0) {
-        float* d = prm.debug + 5 * 48;
+        float* d = prm.debug + 7 * 48;
         d[0] = (float)nch;
         for (int i = 0; i < 12; ++i) d[1 + i] = (float)tt_[i] / nch;
     }
@@ -910,48 +932,6 @@ __device__ void role_chain(const Ctx& cx, const TcParams& prm, int wtid)
             warp_arrive(cx.bar(B_SBF_READY), lane);
             GDN_T(4);
 
-            // ---- output epilogue: O^T = diag(e^G) (S0 Q^T) + Delta^T P^T -------------------------------------
-            // For a fixed token the 128 lanes hold 128 consecutive bf16 of out_o: each warp store writes 64
-            // contiguous bytes (two full sectors), so the outputs go straight from registers to global memory.
-            {
-                __nv_bfloat16* obase = og ? og + ((size_t)row0 * p.Hv + h) * 128 + dv : nullptr;
-                const size_t ostride = (size_t)p.Hv * 128;
-#pragma unroll 1
-                for (int g = 0; g < 2; ++g) {
-                    const int c0 = 32 * hf + 16 * g;
-                    uint32_t a3[16], a2[16];
-                    tmem_ld16(tl + TM_ACC3 + c0, a3);
-                    if (!first) tmem_ld16(tl + TM_ACC2 + c0, a2);
-                    tmem_ld_wait();
-#ifdef GDN_TC_DEBUG
-                    if (dbg) {
-#pragma unroll
-                        for (int i = 0; i < 16; ++i) {
-                            dbase[36864 + dv * 64 + c0 + i] = __uint_as_float(a3[i]);
-                            dbase[28672 + dv * 64 + c0 + i] = !first ? __uint_as_float(a2[i]) : 0.f;
-                        }
-                    }
-#endif
-                    if (og) {
-#pragma unroll
-                        for (int i4 = 0; i4 < 4; ++i4) {
-                            const float4 eg = *reinterpret_cast<const float4*>(&dc.eG[c0 + 4 * i4]);
-                            const float egs[4] = {eg.x, eg.y, eg.z, eg.w};
-#pragma unroll
-                            for (int e = 0; e < 4; ++e) {
-                                const int i = 4 * i4 + e;
-                                float o = __uint_as_float(a3[i]);
-                                if (!first) o = fmaf(egs[e], __uint_as_float(a2[i]), o);
-                                if (c0 + i < nvalid) obase[(size_t)(c0 + i) * ostride] = __float2bfloat16_rn(o);
-                            }
-                        }
-                    }
-                }
-                tc_fence_before();
-                warp_arrive(cx.bar(B_ACC23_FREE), lane);
-                warp_arrive(cx.bar(B_DECAY_FREE0 + (j & 3u)), lane);    // last read of this chunk's decay factors
-                GDN_T(6);
-            }
             GDN_T(8);
             GDN_TIMERS(++nch;)
         }
@@ -969,6 +949,59 @@ __device__ void role_chain(const Ctx& cx, const TcParams& prm, int wtid)
         for (int i = 0; i < 12; ++i) d[1 + i] = (float)tt_[i] / nch;
     }
 #endif
+}
+
+// ================================================================================================
+// warps 23-26: output group (one warp per TMEM lane window).  O^T = diag(e^G) (S0 Q^T) + Delta^T P^T of chunk j,
+// read from the two accumulators as soon as the chunk's last MMAs have completed and stored off the chain's
+// critical path.  For a fixed token the 128 lanes hold 128 consecutive bf16 of out_o: each warp store writes
+// 64 contiguous bytes (two full sectors), so the outputs go straight from registers to global memory.
+// ================================================================================================
+__device__ void role_out(const Ctx& cx, const TcParams& prm, int warp, int lane)
+{
+    const Problem& p = prm.p;
+    const int w4 = warp & 3;
+    const int dv = w4 * 32 + lane;
+    const uint32_t tl = cx.tmem + ((uint32_t)(w4 * 32) << 16);
+    __nv_bfloat16* __restrict__ og = reinterpret_cast<__nv_bfloat16*>(p.out_o);
+    ChunkCursor cc;
+    cc.init(&p, prm.s.order);
+#pragma unroll 1
+    for (uint32_t j = 0; cc.valid; ++j, cc.advance()) {
+        const int row0 = cc.row0(), nvalid = cc.nvalid();
+        const bool first = cc.first();
+        const Decay& dc = cx.misc->decay[j & 3u];
+        cx.wait(B_DECAY_READY0 + (j & 3u), (j >> 2) & 1u);
+        cx.wait(B_MMA3_DONE, j & 1u);
+        tc_fence_after();
+        __nv_bfloat16* optr = og ? og + ((size_t)row0 * p.Hv + cc.h) * 128 + dv : nullptr;
+        const uint32_t ostride = (uint32_t)p.Hv * 128u;
+#pragma unroll 1
+        for (int g = 0; g < 4; ++g) {
+            const int c0 = 16 * g;
+            uint32_t a3[16], a2[16];
+            tmem_ld16(tl + TM_ACC3 + c0, a3);
+            if (!first) tmem_ld16(tl + TM_ACC2 + c0, a2);
+            tmem_ld_wait();
+            if (og) {
+#pragma unroll
+                for (int i4 = 0; i4 < 4; ++i4) {
+                    const float4 eg = *reinterpret_cast<const float4*>(&dc.eG[c0 + 4 * i4]);
+                    const float egs[4] = {eg.x, eg.y, eg.z, eg.w};
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        const int i = 4 * i4 + e;
+                        float o = __uint_as_float(a3[i]);
+                        if (!first) o = fmaf(egs[e], __uint_as_float(a2[i]), o);
+                        if (c0 + i < nvalid) optr[(uint32_t)(c0 + i) * ostride] = __float2bfloat16_rn(o);
+                    }
+                }
+            }
+        }
+        tc_fence_before();
+        warp_arrive(cx.bar(B_ACC23_FREE), lane);
+        warp_arrive(cx.bar(B_DECAY_FREE0 + (j & 3u)), lane);    // last read of this chunk's decay factors
+    }
 }
 
 __global__ void __launch_bounds__(kThreads, 1)
@@ -989,11 +1022,13 @@ gdn_tc_kernel(const TcParams prm, const __grid_constant__ CUtensorMap tm_q,
     }
     if (tid == 32) {
         for (int i = 0; i < NUM_BARS; ++i) {
-            // arrivals per phase: one per warp of the arriving group (8), or of its W^T half (4)
+            // arrivals per phase: one per warp of the arriving group (G1 and chain: 8 warps, G2: 2 warps)
             const bool wg_bar = i == B_GRAM_READ || i == B_TPP_READY || i == B_D_READY || i == B_SBF_READY ||
-                                i == B_ACC23_FREE || (i >= B_DECAY_FREE0 && i <= B_DECAY_FREE3);
-            const bool half_bar = i == B_WACC_READ || i == B_PRE_DONE0 || i == B_PRE_DONE1;
-            mbar_init(cx.bar(i), wg_bar ? (uint32_t)(kWgThreads / 32) : half_bar ? 4u : 1u);
+                                i == B_WACC_READ || i == B_PRE_DONE0 || i == B_PRE_DONE1 ||
+                                i == B_A_READY0 || i == B_A_READY1 || i == B_X_FREE;
+            const bool out_bar = i == B_ACC23_FREE || (i >= B_DECAY_FREE0 && i <= B_DECAY_FREE3);
+            const bool g2_bar = i == B_A_FREE0 || i == B_A_FREE1 || i == B_X_READY;
+            mbar_init(cx.bar(i), wg_bar ? 8u : out_bar ? 4u : g2_bar ? 2u : 1u);
         }
         fence_mbar_init();
         cx.misc->abort = 0u;
@@ -1012,17 +1047,23 @@ gdn_tc_kernel(const TcParams prm, const __grid_constant__ CUtensorMap tm_q,
     } else if (warp == 1) {
         role_mma_chain(cx, prm);
     } else if (warp == 2) {
-        role_mma_pre(cx, prm);
+        role_mma_gram(cx, prm);
     } else if (warp == 3) {
         role_decay(cx, prm);
     } else if (warp >= 4 && warp < 12) {
-        role_pre(cx, prm, tid - 128);
-    } else if (warp >= 12) {
+        role_g1(cx, prm, tid - 128);
+    } else if (warp >= 12 && warp < 20) {
         role_chain(cx, prm, tid - 384);
+    } else if (warp >= 20 && warp < 22) {
+        role_g2(cx, prm, tid - 640);
+    } else if (warp == 22) {
+        role_mma_w(cx, prm);
+    } else if (warp >= 23) {
+        role_out(cx, prm, warp, lane);
     }
 #ifdef GDN_TC_PROFILE
-    if (prm.debug && blockIdx.x == 0 && lane == 0 && (warp < 3 || warp == 4 || warp == 12)) {
-        const int slot = warp < 3 ? warp : (warp == 4 ? 3 : 4);
+    if (prm.debug && blockIdx.x == 0 && lane == 0 && (warp < 3 || warp == 4 || warp == 12 || warp == 20)) {
+        const int slot = warp < 3 ? warp : (warp == 4 ? 3 : (warp == 12 ? 4 : 8));
         cx.prof_dump(prm.debug + slot * 48);
     }
 #endif
