@@ -148,6 +148,16 @@ struct ChunkCursor {
         const uint32_t G = gridDim.x, b = blockIdx.x;
         return (uint32_t)round * G + ((round & 1) ? (G - 1 - b) : b);
     }
+    // Row range and heads of one work item, kept out of line (three integer divisions and two dependent
+    // global loads, needed once per chain by every role): x = first row, y = end row, z = v-head | q/k head << 16,
+    // w = request index.
+    __device__ __noinline__ static int4 lookup(const Problem* p, const int32_t* order, uint32_t item)
+    {
+        const int n = order[item / p->Hv];
+        const int h = item % p->Hv;
+        const int hq = h / (p->Hv / p->Hq);
+        return make_int4(p->cu[n], p->cu[n + 1], h | (hq << 16), n);
+    }
     // moves to the next chain that has at least one chunk
     __device__ void next_chain()
     {
@@ -155,11 +165,8 @@ struct ChunkCursor {
             ++r;
             const uint32_t item = item_of(r);
             if (item >= num_items) { valid = false; return; }
-            n = order[item / p->Hv];
-            h = item % p->Hv;
-            hq = h / (p->Hv / p->Hq);
-            row_begin = p->cu[n];
-            row_end = p->cu[n + 1];
+            const int4 ci = lookup(p, order, item);
+            row_begin = ci.x; row_end = ci.y; h = ci.z & 0xffff; hq = ci.z >> 16; n = ci.w;
             nchunks = (row_end - row_begin + 63) >> 6;
             c = 0;
             if (nchunks > 0) return;
@@ -671,18 +678,18 @@ __device__ void role_g1(const Ctx& cx, const TcParams& prm, int wtid)
     };
 
     if (J == 0) return;
-    post(0);
+    // iteration i: W^T epilogue of chunk i-2 (first: it completes the operand set the chain is waiting for),
+    // Gram post-processing of chunk i (overlaps the solve of chunk i-1), T', T'' of chunk i-1
 #pragma unroll 1
-    for (uint32_t k = 0; k < J; ++k) {
-        if (k >= 1) w_epilogue(k - 1);       // first: it completes the operand set the chain is waiting for
+    for (uint32_t i = 0; i <= J + 1; ++i) {
+        if (i >= 2) w_epilogue(i - 2);
         GDN_T(0);
-        if (k + 1 < J) post(k + 1);          // overlaps the solve of chunk k
+        if (i < J) post(i);
         GDN_T(1);
-        t_write(k);
+        if (i >= 1 && i <= J) t_write(i - 1);
         GDN_T(2);
         GDN_TIMERS(++nch;)
     }
-    w_epilogue(J - 1);
 #ifdef GDN_TC_PROFILE
     if (prm.debug && blockIdx.x == 0 && wtid == 0 && nch > 0) {
         float* d = prm.debug + 5 * 48;
@@ -831,9 +838,9 @@ __device__ void role_chain(const Ctx& cx, const TcParams& prm, int wtid)
     for (int r = 0;; ++r) {
         const uint32_t item = ChunkCursor::item_of(r);
         if (item >= num_items) break;
-        const int n = prm.s.order[item / p.Hv];
-        const int h = item % p.Hv;
-        const int row_begin = p.cu[n], row_end = p.cu[n + 1];
+        const int4 ci = ChunkCursor::lookup(&p, prm.s.order, item);
+        const int n = ci.w, h = ci.z & 0xffff;
+        const int row_begin = ci.x, row_end = ci.y;
         const int nchunks = (row_end - row_begin + 63) >> 6;
         float* st_out = p.out_state ? p.out_state + ((size_t)n * p.Hv + h) * 128 * 128 : nullptr;
         if (nchunks == 0) {                                   // empty request: zero state, no outputs
