@@ -620,7 +620,7 @@ __device__ void role_g1(const Ctx& cx, const TcParams& prm, int wtid)
         // whose completion the W^T epilogue of this iteration has already waited for
         if (k >= 2) cx.wait(B_TP_FREE0 + (k & 1u), ((k >> 1) - 1u) & 1u);
         const int tt = wtid >> 2, q = wtid & 3, c0 = 16 * q;   // row, 16-column quarter
-        uint32_t w1[8], w2[8];
+        float x[16];
 #pragma unroll
         for (int c8 = 0; c8 < 2; ++c8) {
             const uint4 xv = *reinterpret_cast<const uint4*>(XH + (tt * LDA + c0 + 8 * c8) * 2);
@@ -628,22 +628,40 @@ __device__ void role_g1(const Ctx& cx, const TcParams& prm, int wtid)
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
                 const int s0 = c0 + 8 * c8 + 2 * e;
-                const float2 bv = *reinterpret_cast<const float2*>(&dc.beta[s0]);
-                const float2 ev = *reinterpret_cast<const float2*>(&dc.bE[s0]);
-                const float x0 = (s0 <= tt) ? bf_lo(xw[e]) : 0.f, x1 = (s0 + 1 <= tt) ? bf_hi(xw[e]) : 0.f;
-                w1[4 * c8 + e] = pack_bf16x2(x0 * bv.x, x1 * bv.y);
-                w2[4 * c8 + e] = pack_bf16x2(x0 * ev.x, x1 * ev.y);
+                x[8 * c8 + 2 * e] = (s0 <= tt) ? bf_lo(xw[e]) : 0.f;
+                x[8 * c8 + 2 * e + 1] = (s0 + 1 <= tt) ? bf_hi(xw[e]) : 0.f;
             }
         }
         warp_arrive(cx.bar(B_X_FREE), lane);                    // X has been read: the next solve may overwrite it
         const uint32_t o0 = tt * 128 + (((2 * q) ^ (tt & 7)) << 4), o1 = tt * 128 + (((2 * q + 1) ^ (tt & 7)) << 4);
-        uint8_t* tp = cx.sm + SM_TP + (k & 1u) * 8192;
-        *reinterpret_cast<uint4*>(tp + o0) = make_uint4(w1[0], w1[1], w1[2], w1[3]);
-        *reinterpret_cast<uint4*>(tp + o1) = make_uint4(w1[4], w1[5], w1[6], w1[7]);
-        *reinterpret_cast<uint4*>(cx.sm + SM_TPP + o0) = make_uint4(w2[0], w2[1], w2[2], w2[3]);
-        *reinterpret_cast<uint4*>(cx.sm + SM_TPP + o1) = make_uint4(w2[4], w2[5], w2[6], w2[7]);
-        fence_proxy_async_smem();
-        warp_arrive(cx.bar(B_TPP_READY), lane);
+        // T'' first: it is all the W^T MMA waits for, and that MMA then overlaps the T' half of this routine
+        {
+            uint32_t w2[8];
+#pragma unroll
+            for (int i4 = 0; i4 < 4; ++i4) {
+                const float4 ev = *reinterpret_cast<const float4*>(&dc.bE[c0 + 4 * i4]);
+                w2[2 * i4] = pack_bf16x2(x[4 * i4] * ev.x, x[4 * i4 + 1] * ev.y);
+                w2[2 * i4 + 1] = pack_bf16x2(x[4 * i4 + 2] * ev.z, x[4 * i4 + 3] * ev.w);
+            }
+            *reinterpret_cast<uint4*>(cx.sm + SM_TPP + o0) = make_uint4(w2[0], w2[1], w2[2], w2[3]);
+            *reinterpret_cast<uint4*>(cx.sm + SM_TPP + o1) = make_uint4(w2[4], w2[5], w2[6], w2[7]);
+            fence_proxy_async_smem();
+            warp_arrive(cx.bar(B_TPP_READY), lane);
+        }
+        {
+            uint32_t w1[8];
+#pragma unroll
+            for (int i4 = 0; i4 < 4; ++i4) {
+                const float4 bv = *reinterpret_cast<const float4*>(&dc.beta[c0 + 4 * i4]);
+                w1[2 * i4] = pack_bf16x2(x[4 * i4] * bv.x, x[4 * i4 + 1] * bv.y);
+                w1[2 * i4 + 1] = pack_bf16x2(x[4 * i4 + 2] * bv.z, x[4 * i4 + 3] * bv.w);
+            }
+            uint8_t* tp = cx.sm + SM_TP + (k & 1u) * 8192;
+            *reinterpret_cast<uint4*>(tp + o0) = make_uint4(w1[0], w1[1], w1[2], w1[3]);
+            *reinterpret_cast<uint4*>(tp + o1) = make_uint4(w1[4], w1[5], w1[6], w1[7]);
+            // made visible to the tensor core by the proxy fence of this chunk's W^T epilogue, which every
+            // thread executes before the arrival that releases the operand set
+        }
     };
 
     // ---- W^T epilogue of chunk c: bf16 rows [dk][t] as the N-major operand of the S0 W^T MMA; completes the
@@ -655,14 +673,13 @@ __device__ void role_g1(const Ctx& cx, const TcParams& prm, int wtid)
         if (c >= 1) cx.wait(B_MMA1_DONE, (c - 1) & 1u);
         const int drow = w4 * 32 + lane;                        // dk index = TMEM lane
         uint8_t* wrow = cx.sm + SM_WT + drow * 128;
-#pragma unroll 1
-        for (int g = 0; g < 2; ++g) {
-            const int c0 = 32 * hf + 16 * g;
-            uint32_t acc[16];
-            tmem_ld16(tl + TM_WACC + c0, acc);
+        {
+            const int c0 = 32 * hf;
+            uint32_t acc[32];
+            tmem_ld32(tl + TM_WACC + c0, acc);
             tmem_ld_wait();
 #pragma unroll
-            for (int c8 = 0; c8 < 2; ++c8) {
+            for (int c8 = 0; c8 < 4; ++c8) {
                 uint4 u;
                 u.x = pack_bf16x2(__uint_as_float(acc[c8 * 8 + 0]), __uint_as_float(acc[c8 * 8 + 1]));
                 u.y = pack_bf16x2(__uint_as_float(acc[c8 * 8 + 2]), __uint_as_float(acc[c8 * 8 + 3]));
