@@ -164,6 +164,17 @@ GDN_API int64_t tail_select(int64_t prefix_len, double budget_frac);
 /* Static, human-readable text for a gdn_status value. */
 GDN_API const char* gdn_status_string(int32_t status);
 
+/*
+ * Testing aid for the bounded device-side waits (no counterpart in the paper).  Every wait inside the
+ * tensor-core kernel gives up after `wait_timeout_ns` (default 2 s; 0 restores the default), after which the
+ * kernel stops blocking, finishes with unspecified results and writes GDN_ERR_TIMEOUT to desc->status_word.
+ * `skip_kq_load_of_chunk` >= 0 makes each CTA leave out the K/Q tile copy of that chunk of its work list, so
+ * that the wait for it provably runs out (-1, the default, skips nothing).  Nothing faults or hangs: the
+ * point is to exercise the error path with the GPU context staying usable.  Process-wide; not thread-safe
+ * against concurrent forward calls.
+ */
+GDN_API void gdn_test_hooks(uint64_t wait_timeout_ns, int32_t skip_kq_load_of_chunk);
+
 /* Number of kernels the last forward call on this thread enqueued (for launch accounting). */
 GDN_API int32_t gdn_last_launch_count(void);
 

@@ -63,6 +63,8 @@ def load_library():
     lib.gdn_status_string.argtypes = [ctypes.c_int32]
     lib.gdn_last_launch_count.restype = ctypes.c_int32
     lib.gdn_last_launch_count.argtypes = []
+    lib.gdn_test_hooks.restype = None
+    lib.gdn_test_hooks.argtypes = [ctypes.c_uint64, ctypes.c_int32]
     _lib = lib
     return lib
 
@@ -78,6 +80,11 @@ def tail_select(prefix_len: int, budget_frac: float) -> int:
 
 def last_launch_count() -> int:
     return int(load_library().gdn_last_launch_count())
+
+
+def test_hooks(wait_timeout_ns: int = 0, skip_kq_load_of_chunk: int = -1) -> None:
+    """Testing aid: bound of the device-side waits and an optional K/Q tile copy to leave out (see the header)."""
+    load_library().gdn_test_hooks(int(wait_timeout_ns), int(skip_kq_load_of_chunk))
 
 
 def workspace_size(desc: GdnDesc) -> int:

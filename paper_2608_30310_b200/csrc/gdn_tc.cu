@@ -82,6 +82,7 @@ struct Misc {
     unsigned long long bars[NUM_BARS];
     uint32_t tmem_base;
     volatile uint32_t abort;
+    unsigned long long timeout_ns;
 };
 constexpr uint32_t SM_TOTAL = SM_MISC + ((sizeof(Misc) + 1023) / 1024) * 1024;
 constexpr uint32_t SMEM_BYTES = SM_TOTAL + 1024;   // slack for the manual 1024-byte alignment
@@ -111,7 +112,9 @@ constexpr uint32_t ID_DK = idesc_bf16(128, 128, 0, 1, 0);     // Delta'^T (TMEM)
 struct TcParams {
     Problem p;
     Sched s;
-    float* debug;     // debug builds only: intermediates of the first chain's first two chunks
+    float* debug;                 // debug builds only: intermediates of the first chain's first two chunks
+    unsigned long long wait_timeout_ns;   // bound of every device-side wait
+    int32_t skip_kq_load;         // testing aid: chunk whose K/Q copy is left out (-1: none)
 };
 
 #ifdef GDN_TC_DEBUG
@@ -225,7 +228,7 @@ struct Ctx {
             // suspended in hardware until the phase completes (or ~20 us pass): no polling instructions
             if (mbar_try_wait_hint(b, parity, 20000u)) return true;
             if (misc->abort) return true;
-            if (globaltimer_ns() - t0 > 2000000000ull) { misc->abort = 1u; return true; }
+            if (globaltimer_ns() - t0 > misc->timeout_ns) { misc->abort = 1u; return true; }
         }
     }
 };
@@ -310,6 +313,7 @@ __device__ void role_producer(const Ctx& cx, const TcParams& prm, const CUtensor
     cv = ckq;
     auto load_kq = [&](const ChunkCursor& cc, uint32_t j) {
         const uint32_t slot = j % 3u, dst = cx.sb + SM_KQ + slot * KQ_SLOT, bar = cx.bar(B_FULL_KQ0 + slot);
+        if ((int32_t)j == prm.skip_kq_load) return;       // testing aid: this tile never arrives
         if (elect_one()) {
             mbar_arrive_expect_tx(bar, 32768u);
             tma_load_2d(dst, tm_k, cc.hq * 128, cc.row0(), bar);
@@ -1056,6 +1060,7 @@ gdn_tc_kernel(const TcParams prm, const __grid_constant__ CUtensorMap tm_q,
         }
         fence_mbar_init();
         cx.misc->abort = 0u;
+        cx.misc->timeout_ns = prm.wait_timeout_ns;
         prefetch_tmap(&tm_q); prefetch_tmap(&tm_k); prefetch_tmap(&tm_v);
     }
     tc_fence_before();
@@ -1136,12 +1141,20 @@ bool make_map(CUtensorMap* m, const void* base, uint64_t rows, uint64_t cols)
 }
 
 float* g_debug_buffer = nullptr;
+unsigned long long g_wait_timeout_ns = 2000000000ull;
+int32_t g_skip_kq_load = -1;
 
 }  // namespace
 
 #if defined(GDN_TC_DEBUG) || defined(GDN_TC_PROFILE)
 extern "C" GDN_API void gdn_debug_set_buffer(float* dev_ptr) { g_debug_buffer = dev_ptr; }
 #endif
+
+extern "C" GDN_API void gdn_test_hooks(uint64_t wait_timeout_ns, int32_t skip_kq_load_of_chunk)
+{
+    g_wait_timeout_ns = wait_timeout_ns ? wait_timeout_ns : 2000000000ull;
+    g_skip_kq_load = skip_kq_load_of_chunk;
+}
 
 cudaError_t launch_tcgen05(const Problem& p, const Sched& s, cudaStream_t stream, int* launches)
 {
@@ -1166,6 +1179,7 @@ cudaError_t launch_tcgen05(const Problem& p, const Sched& s, cudaStream_t stream
     if (grid > sms) grid = sms;
     TcParams prm;
     prm.p = p; prm.s = s; prm.debug = g_debug_buffer;
+    prm.wait_timeout_ns = g_wait_timeout_ns; prm.skip_kq_load = g_skip_kq_load;
     gdn_tc_kernel<<<(unsigned)grid, kThreads, SMEM_BYTES, stream>>>(prm, tq, tk, tv);
     e = cudaGetLastError();
     if (e == cudaSuccess && launches) *launches += 1;
