@@ -14,7 +14,6 @@ import argparse
 import json
 import os
 import statistics
-import subprocess
 import sys
 import threading
 import time
@@ -33,9 +32,10 @@ WORKLOAD = "concurrent_hits_32req_tails_U400-3300_Hq16_Hv32_d128_bf16_chunk64"
 BYTES_PER_TOKEN_HEAD = 776.0        # q,k shared by 2 v-heads + v + o in bf16, g and beta in fp32
 FLOPS_PER_TOKEN_HEAD = 139264.0     # 6 dk dv + C (3 dk + 2 dv), triangular products at half cost
 STATE_BYTES_PER_CHAIN = 128 * 128 * 4
-# DRAM bytes per token*head of the dominant kernel from the committed ncu capture (profiles/),
-# scaled to a launch by the units it processes; None until a capture exists.
-NCU_TRAFFIC_BYTES_PER_TOKEN_HEAD = None
+# DRAM bytes per token*head of the dominant kernel, from the committed ncu capture of the 8-request case
+# (profiles/gdn_tc_kernel_concurrent_hits_8req.md: dram read + write = 272.1 MB for 346,944 token*heads,
+# final states included); traffic grows in proportion to the units a launch processes.
+NCU_TRAFFIC_BYTES_PER_TOKEN_HEAD = 784.4
 
 
 def load_peaks():
@@ -47,57 +47,58 @@ def load_peaks():
 
 
 class ClockSampler:
-    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
-    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
-              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
-              "clocks_event_reasons.sw_power_cap")
+    """Samples SM clocks and throttle reasons through NVML (read-only) in a thread while the timed region runs."""
+    REASONS = {0x4: "sw_power_cap", 0x8: "hw_slowdown", 0x20: "sw_thermal_slowdown", 0x40: "hw_thermal_slowdown"}
 
-    def __init__(self, index: int):
-        self.index = index
-        self.rows = []
-        self.proc = None
+    def __init__(self, cuda_index: int):
+        self.cuda_index = cuda_index
+        self.sm = []
+        self.reasons = set()
+        self.sm_max = None
+        self.stop_flag = False
         self.thread = None
+        self.handle = None
+        try:
+            import pynvml
+            import torch
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            try:
+                uuid = str(torch.cuda.get_device_properties(cuda_index).uuid)
+                if not uuid.startswith("GPU-"):
+                    uuid = "GPU-" + uuid
+                self.handle = pynvml.nvmlDeviceGetHandleByUUID(uuid.encode())
+            except Exception:
+                self.handle = pynvml.nvmlDeviceGetHandleByIndex(cuda_index)
+            self.sm_max = float(pynvml.nvmlDeviceGetMaxClockInfo(self.handle, pynvml.NVML_CLOCK_SM))
+        except Exception:
+            self.handle = None
+
+    def _poll(self):
+        nv = self.nv
+        while not self.stop_flag:
+            try:
+                self.sm.append(float(nv.nvmlDeviceGetClockInfo(self.handle, nv.NVML_CLOCK_SM)))
+                mask = int(nv.nvmlDeviceGetCurrentClocksEventReasons(self.handle))
+                for bit, name in self.REASONS.items():
+                    if mask & bit:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            time.sleep(0.001)
 
     def start(self):
-        try:
-            self.proc = subprocess.Popen(
-                ["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.FIELDS,
-                 "--format=csv,noheader,nounits", "-lms", "100"],
-                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
-        except OSError:
-            self.proc = None
+        if self.handle is None:
             return
-        self.thread = threading.Thread(target=self._read, daemon=True)
+        self.thread = threading.Thread(target=self._poll, daemon=True)
         self.thread.start()
 
-    def _read(self):
-        for line in self.proc.stdout:
-            parts = [x.strip() for x in line.split(",")]
-            if len(parts) >= 7:
-                self.rows.append(parts)
-
     def stop(self):
-        if self.proc is not None:
-            self.proc.terminate()
-            try:
-                self.proc.wait(timeout=5)
-            except Exception:
-                self.proc.kill()
-        sm = []
-        smax = None
-        reasons = set()
-        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for r in self.rows:
-            try:
-                sm.append(float(r[0]))
-                smax = float(r[1])
-            except ValueError:
-                continue
-            for nm, val in zip(names, r[3:7]):
-                if val.lower().startswith("active"):
-                    reasons.add(nm)
-        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": smax,
-                "reasons": sorted(reasons), "samples": len(sm)}
+        self.stop_flag = True
+        if self.thread is not None:
+            self.thread.join(timeout=2)
+        return {"sm_mhz": statistics.median(self.sm) if self.sm else None, "sm_max_mhz": self.sm_max,
+                "reasons": sorted(self.reasons), "samples": len(self.sm)}
 
 
 def to_device(inp, device):
@@ -141,6 +142,21 @@ def oracle_timed(inp, budget_s=20.0):
     sample = "first %d of %d requests (%d tokens x %d heads), fp64 token-by-token, %.1f s" % (
         take, len(lens), tok, Hv, dt)
     return {"value": tok * Hv / dt, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample}, dt
+
+
+def reduce_over_ranks(elapsed_ms: float, units: float, device="cpu"):
+    """Whole-job view of one timed region: MAX of the elapsed time and SUM of the processed units over all
+    ranks (identity when torch.distributed is not initialised).  The path has no exchange step, so this
+    reduction of two scalars is the only collective of a multi-GPU run and it sits outside the timed region."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return float(elapsed_ms), float(units)
+    t = torch.tensor([float(elapsed_ms)], dtype=torch.float64, device=device)
+    u = torch.tensor([float(units)], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    dist.all_reduce(u, op=dist.ReduceOp.SUM)
+    return float(t.item()), float(u.item())
 
 
 def run_reference(args, rank):
@@ -241,16 +257,10 @@ def main():
     total_ms = e0.elapsed_time(e1)
     call_ms = [a.elapsed_time(b) for a, b in evs]
     clocks = sampler.stop()
-    t = torch.tensor([total_ms], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    total_ms = float(t.item())
-    ms_per_step = total_ms / args.steps
     units_per_step = T * Hv
-    tu = torch.tensor([float(units_per_step)], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(tu, op=dist.ReduceOp.SUM)
-    value = float(tu.item()) / (ms_per_step * 1e-3)
+    total_ms, units_all = reduce_over_ranks(total_ms, units_per_step, dev)
+    ms_per_step = total_ms / args.steps
+    value = units_all / (ms_per_step * 1e-3)
 
     # roofline of the dominant kernel (the chunkwise forward); each call = a ~2 us scheduler kernel
     # + this kernel, timed together with events on the launching stream, so `achieved` is a floor
@@ -295,12 +305,10 @@ def main():
             step_host()
         b.record(stream)
         barrier()
-        te = torch.tensor([a.elapsed_time(b)], dtype=torch.float64, device=dev)
-        if world > 1:
-            dist.all_reduce(te, op=dist.ReduceOp.MAX)
-        e2e = {"value": float(tu.item()) / (float(te.item()) / e2e_steps * 1e-3), "unit": UNIT,
+        te, _ = reduce_over_ranks(a.elapsed_time(b), units_per_step, dev)
+        e2e = {"value": units_all / (te / e2e_steps * 1e-3), "unit": UNIT,
                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps,
-               "ms_per_step": float(te.item()) / e2e_steps}
+               "ms_per_step": te / e2e_steps}
         del hq, hk, hv_, ho, hs
 
     # us per 32K-hit state rebuild: 36 GDN layers back to back, batch 1, 5 % and 10 % budgets
@@ -342,10 +350,10 @@ def main():
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
-            "scaling": "weak", "vs_baseline": None, "dtype": "bf16 in/out, fp32 accumulate and state",
+            "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
             "data": "synthetic",
             "config": {"workload": WORKLOAD, "requests": N, "tokens": T, "v_heads": Hv, "qk_heads": inp.num_qk_heads,
-                       "chunk": 64, "l2": "inputs per step (1.5 GB) exceed L2, no flush",
+                       "chunk": 64, "state": "fp32", "l2": "inputs per step (1.5 GB) exceed L2, no flush",
                        "kernel": {0: "auto", 1: "fp32_simt", 2: "tcgen05"}[args.kernel]},
             "roofline": roofline, "cpu_baseline": cpu_baseline, "e2e": e2e, "clocks": clocks,
             "gpu_launches": launches_per_step * args.steps,
