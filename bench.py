@@ -186,6 +186,72 @@ def run_reference(args, rank):
     print(json.dumps(line), flush=True)
 
 
+def run_sweep(args, dev, gdn):
+    """Timings of the other named configurations on one GPU (CUDA events, 3 warm-ups + 10 repetitions, 256 MB
+    L2 flush before every repetition, 4 rotating seeded input sets where a configuration has layers)."""
+    import torch
+    from gdn_workloads import config_single_layer, config_full_prefill
+    stream = torch.cuda.current_stream()
+    ws = gdn.Workspace(dev)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+
+    def timed(call, reps=10, warm=3):
+        ts = []
+        for r in range(warm + reps):
+            flush.zero_()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            call()
+            b.record(stream)
+            torch.cuda.synchronize()
+            if r >= warm:
+                ts.append(a.elapsed_time(b) * 1e3)
+        return {"us_mean": statistics.mean(ts), "us_min": min(ts)}
+
+    def layer_sets(make, n=4):
+        return [to_device(make(i), dev) for i in range(n)]
+
+    out = {}
+    sets = layer_sets(lambda i: config_single_layer(seed_offset=i))
+    L = 1638
+    oo = torch.empty((L, 32, 128), dtype=torch.bfloat16, device=dev)
+    ss = torch.empty((1, 32, 128, 128), dtype=torch.float32, device=dev)
+    it = [0]
+
+    def one_layer():
+        x = sets[it[0] % 4]
+        it[0] += 1
+        gdn.gdn_tail_replay(x[0], x[1], x[2], x[3], x[4], x[5], 64, oo, ss, workspace=ws, kernel=args.kernel, stream=stream)
+    r = timed(one_layer)
+    r["tokens_heads_per_s"] = L * 32 / (r["us_mean"] * 1e-6)
+    out["single_layer_tail_1638"] = r
+    del sets
+    for cfg in config_budget_sweep_tails():
+        L = cfg["tail"]
+        sets = layer_sets(lambda i: config_budget_sweep_layer(L, layer=i))
+        oo = torch.empty((L, 32, 128), dtype=torch.bfloat16, device=dev)
+
+        def rebuild():
+            for layer in range(36):
+                x = sets[layer % 4]
+                gdn.gdn_tail_replay(x[0], x[1], x[2], x[3], x[4], x[5], 64, oo, ss, workspace=ws, kernel=args.kernel, stream=stream)
+        r = timed(rebuild)
+        r["layers"] = 36
+        out["rebuild_prefix_%d_budget_%d%%_tail_%d" % (cfg["prefix"], cfg["budget_pct"], L)] = r
+        del sets
+    for m in (32768, 131072):
+        x = to_device(config_full_prefill(m), dev)
+        oo = torch.empty((m, 32, 128), dtype=torch.bfloat16, device=dev)
+
+        def prefill():
+            gdn.gdn_full_prefill(x[0], x[1], x[2], x[3], x[4], x[5], 64, oo, ss, workspace=ws, kernel=args.kernel, stream=stream)
+        r = timed(prefill, reps=5)
+        r["tokens_heads_per_s"] = m * 32 / (r["us_mean"] * 1e-6)
+        out["full_prefill_%d" % m] = r
+        del x, oo
+    print(json.dumps({"sweep": out, "unit": "us", "n_gpus": 1, "dtype": "bf16", "data": "synthetic"}), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -196,6 +262,9 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--requests", type=int, default=32, help="requests in the batch (32 = the named workload)")
+    ap.add_argument("--sweep", action="store_true",
+                    help="instead of the benchmark line, time the other named configurations (single layer, "
+                         "budget sweep x 36 layers, full prefill 32K / 128K) and print them as one JSON line")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
@@ -218,6 +287,10 @@ def main():
     if world > 1:
         dist.init_process_group("nccl", device_id=dev)
     gdn.load_library()
+
+    if args.sweep:
+        run_sweep(args, dev, gdn)
+        return
 
     # every rank replays its own batch (weak scaling); seeds differ per rank
     inp = config_concurrent_hits(num_seqs=args.requests, seed_offset=rank)

@@ -168,6 +168,16 @@ def test_config4_full_prefill_and_alpha_product_bound(kernel):
 
 
 @pytest.mark.parametrize("kernel", [TC])
+def test_config4_full_prefill_128k_sampled(kernel):
+    """The largest named size: zero-state forward over a 131,072-token prefix (2,048 serial chunks per head);
+    one whole chain is checked against the oracle, every state for finiteness."""
+    full = config_full_prefill(131072)
+    o, st, _ = run_library(full, kernel=kernel, fn="gdn_full_prefill")
+    assert np.isfinite(st).all()
+    _sampled_chain_parity(full, o, st, [(0, 5)])
+
+
+@pytest.mark.parametrize("kernel", [TC])
 def test_weak_decay_tail_vs_full_bound_has_teeth(kernel):
     full = config_full_prefill(600, g_lo=-0.002, g_hi=-0.0001, num_qk_heads=2, num_v_heads=4)
     _, st, _ = run_library(full, kernel=kernel)
