@@ -804,27 +804,29 @@ __device__ void role_g2(const Ctx& cx, const TcParams& prm, int wtid)
         }
         pair_sync();
         GDN_T(1);
-        // level 2: warp pw owns block row mt = pw of X[32:64][0:32], both block columns
+        // level 2: warp pw owns block row mt = pw of X[32:64][0:32]; its two 16 x 16 tiles are independent, so
+        // their ldmatrix / mma chains are written side by side to overlap their latencies
         {
             const int mt = pw;
-#pragma unroll 1
-            for (int nt = 0; nt < 2; ++nt) {
-                float m[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
-                // X11 is lower triangular: block column nt starts at block row nt
-                for (int kb = nt; kb < 2; ++kb)
-                    tile16_mma(m, ah, LDA, 32 + 16 * mt, 16 * kb, xh, LDA, 16 * kb, 16 * nt, lane);
-                tile16_store(m, 1.f, MH, LDM, 16 * mt, 16 * nt, lane);
-            }
+            float m0[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}}, m1[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
+            // X11 is lower triangular: block column nt starts at block row nt
+            tile16_mma(m0, ah, LDA, 32 + 16 * mt, 0, xh, LDA, 0, 0, lane);
+            tile16_mma(m1, ah, LDA, 32 + 16 * mt, 16, xh, LDA, 16, 16, lane);
+            tile16_mma(m0, ah, LDA, 32 + 16 * mt, 16, xh, LDA, 16, 0, lane);
+            tile16_store(m0, 1.f, MH, LDM, 16 * mt, 0, lane);
+            tile16_store(m1, 1.f, MH, LDM, 16 * mt, 16, lane);
             warp_arrive(cx.bar(B_A_FREE0 + (k & 1u)), lane);   // last read of this chunk's A
             pair_sync();
-#pragma unroll 1
-            for (int nt = 0; nt < 2; ++nt) {
-                float d[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
-                // X22 is lower triangular: block row mt ends at block column mt
-                for (int kb = 0; kb <= mt; ++kb)
-                    tile16_mma(d, xh, LDA, 32 + 16 * mt, 32 + 16 * kb, mh, LDM, 16 * kb, 16 * nt, lane);
-                tile16_store(d, -1.f, XH, LDA, 32 + 16 * mt, 16 * nt, lane);
+            float d0[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}}, d1[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
+            // X22 is lower triangular: block row mt ends at block column mt
+            tile16_mma(d0, xh, LDA, 32 + 16 * mt, 32, mh, LDM, 0, 0, lane);
+            tile16_mma(d1, xh, LDA, 32 + 16 * mt, 32, mh, LDM, 0, 16, lane);
+            if (mt == 1) {
+                tile16_mma(d0, xh, LDA, 48, 48, mh, LDM, 16, 0, lane);
+                tile16_mma(d1, xh, LDA, 48, 48, mh, LDM, 16, 16, lane);
             }
+            tile16_store(d0, -1.f, XH, LDA, 32 + 16 * mt, 0, lane);
+            tile16_store(d1, -1.f, XH, LDA, 32 + 16 * mt, 16, lane);
         }
         warp_arrive(cx.bar(B_X_READY), lane);
         GDN_T(2);
