@@ -8,13 +8,17 @@
 //   G_t   = cumsum(g) inside the chunk;  Gam[t,s] = exp(G_t - G_s) (t >= s)
 //   Gram  = [K;Q] K^T                        (MMA, 128 x 64: rows 0-63 K K^T, rows 64-127 Q K^T)
 //   A     = strict_lower(beta_t Gam (K K^T)),  P = lower_incl(Gam (Q K^T))
-//   X     = (I + A)^-1                        (16 x 16 diagonal blocks by substitution in fp32, block
-//                                              merges on mma.sync bf16 with ldmatrix-fed fragments)
-//   T'    = X diag(beta),  T'' = X diag(beta e^G)
-//   W^T   = K^T T''^T                         (MMA, 128(dk) x 64)
-//   Dl^T  = V^T T'^T - S0 W^T                 (two MMAs into one accumulator, second negated)
+//   X     = (I + A)^-1,  T' = X diag(beta),  T'' = X diag(beta e^G).  With beta moved to the columns,
+//   A^    = strict_lower(Gam (K K^T)) diag(beta) and P^ = (I + A^)^-1 (8 x 8 diagonal blocks by substitution
+//           in fp32, block merges on mma.sync bf16 with ldmatrix-fed fragments), one has T' = diag(beta) P^ and
+//           T'' = diag(beta) P^ diag(e^G): P^ itself and its column-scaled copy P^ diag(e^G) are the two MMA
+//           operands, and the common row factor beta is applied in the Delta epilogue
+//   W~^T  = K^T (P^ diag(e^G))^T              (MMA, 128(dk) x 64)
+//   Dl^T  = (V^T P^^T - S0 W~^T) diag(beta)   (two MMAs into one accumulator, second negated)
 //   O^T   = (S0 Q^T) diag(e^G) + Dl^T P^T     (two MMAs, combined in the epilogue)
-//   S     = e^{G_C} S0 + (Dl diag(e^{G_C - G}))^T K    (MMA accumulating onto the pre-scaled state)
+//   S     = e^{G_C} S0 + (Dl diag(e^{G_C - G}))^T K    (MMA accumulating in place: tensor memory holds S / c with
+//                                              c the running product of the chunk decays, folded into the
+//                                              per-token factors; rescaled before c drops below 2^-40)
 //
 // The CTA is warp-specialised and software-pipelined over the chunks of all chains it owns (27 warps):
 //   warp 0       TMA producer: K/Q tiles two chunks ahead (3 slots), V one chunk ahead (1 slot)
@@ -22,10 +26,11 @@
 //   warp 2       issues the Gram MMAs, two chunks ahead of the chain
 //   warp 3       decay warp: loads g and beta up to three chunks ahead, scans the log-decay and publishes the
 //                per-chunk decay factors
-//   warps 4-11   group G1 (two warps per TMEM lane window): Gram post-processing (A, P) of chunk k+1, then
-//                T', T'' of chunk k once its inverse is ready, and the W^T epilogue of chunk k-1
-//   warps 12-19  chain group: Delta epilogue, state conversion and pre-scaling, final state (chunk j)
-//   warps 20-21  group G2: the triangular solve of chunk k, overlapped with G1's other work
+//   warps 4-11   group G1 (two warps per TMEM lane window): Gram post-processing (A^, P) of chunk k+1, then the
+//                W^T epilogue of chunk k
+//   warps 12-19  chain group: Delta epilogue, state conversion (and rescaling when due), final state (chunk j)
+//   warps 20-21  group G2: the triangular solve of chunk k, built in place in the T' operand buffer, with the
+//                column-scaled copy written to the T'' operand buffer block by block
 //   warp 22      issues the W^T MMAs
 //   warps 23-26  output group: output epilogue of chunk j, off the chain's critical path
 // Every per-chunk loop is kept rolled with 16-column TMEM accesses: straight-line code larger than the
@@ -56,28 +61,37 @@ constexpr uint32_t KQ_SLOT = 32768;
 constexpr uint32_t SM_V = 98304;              // 2 halves x [64 rows] x 128 B                               16 KB
 constexpr uint32_t SM_WT = 114688;            // W^T [dk][t] bf16, 128 rows x 128 B                          16 KB
 constexpr uint32_t SM_TP = 131072;            // 2 x T'  [t][s] bf16                                        16 KB
-constexpr uint32_t SM_TPP = 147456;           // T'' [t][s] bf16                                             8 KB
-constexpr uint32_t SM_P = 155648;             // 3 x P [t][s] bf16                                          24 KB
-constexpr uint32_t SM_AH = 180224;            // 2 x A bf16 [64][LDA]
+constexpr uint32_t SM_TPP = 147456;           // 2 x T'' [t][s] bf16                                        16 KB
+constexpr uint32_t SM_P = 163840;             // 3 x P [t][s] bf16                                          24 KB
+constexpr uint32_t SM_AH = 188416;            // 2 x A bf16 [64][LDA]
 constexpr uint32_t AH_BYTES = 64 * LDA * 2;
-constexpr uint32_t SM_XH = SM_AH + 2 * AH_BYTES;   // X = (I + A)^-1 bf16 [64][LDA]
-constexpr uint32_t SM_MH = SM_XH + 64 * LDA * 2;   // merge scratch bf16 [32][LDM]
+constexpr uint32_t SM_MH = SM_AH + 2 * AH_BYTES;   // merge scratch of the solve, bf16 [32][LDM]
 constexpr uint32_t SM_MISC = ((SM_MH + 32 * LDM * 2 + 1023) / 1024) * 1024;
 
 enum Bar {
-    B_FULL_KQ0 = 0, B_FULL_KQ1, B_FULL_KQ2, B_FULL_V, B_GRAM_DONE, B_W_DONE, B_U_DONE, B_MMA1_DONE,
+    B_FULL_KQ0 = 0, B_FULL_KQ1, B_FULL_KQ2, B_FULL_V, B_GRAM_DONE, B_W_DONE0, B_W_DONE1, B_U_DONE, B_MMA1_DONE,
     B_MMA3_DONE, B_KQ_FREE0, B_KQ_FREE1, B_KQ_FREE2, B_P_FREE0, B_P_FREE1, B_P_FREE2, B_TP_FREE0, B_TP_FREE1,
     B_GRAM_READ, B_WACC_READ, B_TPP_READY,
     B_PRE_DONE0, B_PRE_DONE1, B_D_READY, B_SBF_READY, B_ACC23_FREE,
     B_DECAY_READY0, B_DECAY_READY1, B_DECAY_READY2, B_DECAY_READY3,
     B_DECAY_FREE0, B_DECAY_FREE1, B_DECAY_FREE2, B_DECAY_FREE3,
-    B_A_READY0, B_A_READY1, B_A_FREE0, B_A_FREE1, B_X_READY, B_X_FREE, NUM_BARS
+    B_A_READY0, B_A_READY1, B_A_FREE0, B_A_FREE1, B_TP_READY0, B_TP_READY1, NUM_BARS
 };
 
-// G2 = log2(e) * cumulative log-decay; bE = beta e^G; eG = e^G; eRest = e^{G_C - G}
 // colf[s] = 2^(G2_31 - G2_s), s < 32: column factors of the purely off-diagonal quadrant of Gam
-struct Decay { float G2[64], beta[64], bE[64], eG[64], eRest[64], colf[32]; float eGC; float G2mid; float pad[2]; };
+// Per-chunk decay factors.  The fp32 state lives in tensor memory divided by a running factor c (the product of
+// the chunk decays since the last rescale), so that a chunk update is a plain accumulation; c is folded into
+// the factors below, and the state is rescaled (c back to 1) before c leaves [2^-40, 1].
+//   G2    log2-domain inclusive cumulative decay,  beta
+//   colf  2^(G2[31] - G2[s]) for s < 32,  colfb = colf * beta[s]
+//   eG    e^G c_prev         (column factors of T'', so that W^T comes out multiplied by c_prev, as
+//                             S0 = c_prev * stored state; also the output epilogue's factor of (stored state) q)
+//   bRest beta e^(G_C - G) / c   (Delta' = Delta~ diag(bRest) accumulates onto the stored state)
+//   rescale / wb: this chunk starts from a rescaled state: the previous chunk's state epilogue multiplies the
+//   stored state by wb = c_prev e^(G_C) first;  cfin = c after this chunk (final state = cfin * stored state)
+struct Decay { float G2[64], beta[64], eG[64], bRest[64], colf[32], colfb[32]; float wb; float G2mid; float cfin; int rescale; };
 struct Misc {
+    float ones[64];
     Decay decay[4];                    // per-chunk decay factors, ring of 4 (decay warp writes; pre and chain read)
     unsigned long long bars[NUM_BARS];
     uint32_t tmem_base;
@@ -191,6 +205,7 @@ struct Ctx {
     Misc* misc;
     uint32_t tmem;
     __device__ uint32_t bar(int i) const { return sb + SM_MISC + (uint32_t)offsetof(Misc, bars) + 8u * i; }
+    __device__ bool stop() const { return __shfl_sync(0xffffffffu, misc->abort, 0) != 0u; }
     // Bounded wait.  On expiry it raises the CTA-wide abort flag; from then on no wait blocks any more, so
     // every role still runs through its (data-independent) loop structure, keeps meeting its warpgroup
     // barriers and reaches the end of the kernel; the results are garbage and the host sees the status word.
@@ -264,6 +279,25 @@ __device__ __forceinline__ void mma_bf16(float (&c)[4], const uint32_t (&a)[4], 
                  : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
                  : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
+// same four 8 x 8 matrices of a 64 x 64 bf16 tile kept in MMA operand layout: 128-byte rows, 16-byte chunk
+// index XORed with (row & 7)
+__device__ __forceinline__ uint32_t sw_off(int row, int col)
+{
+    return (uint32_t)(row * 128 + ((((col >> 3) ^ (row & 7))) << 4) + (col & 7) * 2);
+}
+__device__ __forceinline__ uint32_t tile_addr_sw(uint32_t base, int row0, int col0, int lane)
+{
+    return base + sw_off(row0 + (lane & 7) + ((lane >> 3) & 1) * 8, col0 + (lane >> 4) * 8);
+}
+// c (16 x 16, two 8-column halves) += A tile * B tile, each given by its per-lane ldmatrix address
+__device__ __forceinline__ void tile16_mma_at(float (&c)[2][4], uint32_t a_addr, uint32_t b_addr)
+{
+    uint32_t a[4], b[4];
+    ldm_x4(a, a_addr);
+    ldm_x4_trans(b, b_addr);
+    mma_bf16(c[0], a, b[0], b[1]);
+    mma_bf16(c[1], a, b[2], b[3]);
+}
 // c (16 x 16, two 8-column halves) += A[ar0.., ak0..+16) * B[bk0..+16, bn0..+16)
 __device__ __forceinline__ void tile16_mma(float (&c)[2][4], uint32_t a_base, int lda, int ar0, int ak0,
                                            uint32_t b_base, int ldb, int bk0, int bn0, int lane)
@@ -326,7 +360,7 @@ __device__ void role_producer(const Ctx& cx, const TcParams& prm, const CUtensor
     uint32_t jkq = 0;
     for (; jkq < 2 && ckq.valid; ++jkq) { load_kq(ckq, jkq); ckq.advance(); }
 #pragma unroll 1
-    for (uint32_t j = 0; cv.valid; ++j) {
+    for (uint32_t j = 0; cv.valid && !cx.stop(); ++j) {
         // V(j): the single slot is free once U^T MMA of chunk j-1 has completed
         if (j >= 1) cx.wait(B_U_DONE, (j - 1) & 1u);
         const uint32_t bar = cx.bar(B_FULL_V);
@@ -383,10 +417,10 @@ __device__ void role_mma_w(const Ctx& cx, const TcParams& prm)
 {
     ChunkCursor cc;
     cc.init(&prm.p, prm.s.order);
-    const uint64_t d_tpp = smem_desc_sw128(cx.sb + SM_TPP, 16, 1024);
 #pragma unroll 1
     for (uint32_t j = 0; cc.valid; ++j, cc.advance()) {
         const uint64_t d_kt = smem_desc_sw128(cx.sb + SM_KQ + (j % 3u) * KQ_SLOT, 16384, 1024);   // K^T, M-major
+        const uint64_t d_tpp = smem_desc_sw128(cx.sb + SM_TPP + (j & 1u) * 8192, 16, 1024);
         cx.wait(B_TPP_READY, j & 1u);
         if (j >= 1) cx.wait(B_WACC_READ, (j - 1) & 1u);
         tc_fence_after();
@@ -394,7 +428,7 @@ __device__ void role_mma_w(const Ctx& cx, const TcParams& prm)
 #pragma unroll
             for (int ks = 0; ks < 4; ++ks)
                 mma_ss(cx.tmem + TM_WACC, desc_add(d_kt, ks * 2048), desc_add(d_tpp, ks * 32), ID_WU, ks > 0);
-            mma_commit(cx.bar(B_W_DONE));
+            mma_commit(cx.bar(B_W_DONE0 + (j & 1u)));
         }
         __syncwarp();
     }
@@ -418,6 +452,7 @@ __device__ void role_mma_chain(const Ctx& cx, const TcParams& prm)
         const uint64_t d_tp = smem_desc_sw128(cx.sb + SM_TP + (j & 1u) * 8192, 16, 1024);
         const bool first = cc.first();
         cx.wait(B_PRE_DONE0 + (j & 1u), (j >> 1) & 1u);
+        cx.wait(B_TP_READY0 + (j & 1u), (j >> 1) & 1u);
         cx.wait(B_FULL_V, j & 1u);
         tc_fence_after();
         // U^T = V^T T'^T -> ACC1 (free: the Delta epilogue of chunk j-1 came before that chunk's last MMAs)
@@ -478,6 +513,7 @@ __device__ void role_decay(const Ctx& cx, const TcParams& prm)
     const int lane = threadIdx.x & 31;
     ChunkCursor cc;
     cc.init(&p, prm.s.order);
+    float c = 1.f;                                            // running scale of the stored state (see Decay)
 #pragma unroll 1
     for (uint32_t j = 0; cc.valid; ++j, cc.advance()) {
         const int row0 = cc.row0(), nvalid = cc.nvalid(), h = cc.h;
@@ -494,18 +530,23 @@ __device__ void role_decay(const Ctx& cx, const TcParams& prm)
         }
         G1 += __shfl_sync(0xffffffffu, G0, 31);
         const float GC = __shfl_sync(0xffffffffu, G1, 31);
-        const float e0 = ex2_approx(G0), e1 = ex2_approx(G1);
+        const float cprev = cc.first() ? 1.f : c;
+        const float eGC = ex2_approx(GC);
+        const bool rescale = cc.first() || !(cprev * eGC >= 9.094947e-13f);       // 2^-40; also catches NaN
+        c = rescale ? 1.f : cprev * eGC;
+        const float cinv = rescale ? 1.f : __frcp_rn(c);
+        const float e0 = ex2_approx(G0) * cprev, e1 = ex2_approx(G1) * cprev;
         // the slot was last read by the chain group's output epilogue of chunk j - 4
         if (j >= 4) cx.wait(B_DECAY_FREE0 + (j & 3u), ((j >> 2) - 1u) & 1u);
         Decay& dc = cx.misc->decay[j & 3u];
         dc.G2[lane] = G0; dc.G2[lane + 32] = G1;
         dc.beta[lane] = b0; dc.beta[lane + 32] = b1;
-        dc.bE[lane] = b0 * e0; dc.bE[lane + 32] = b1 * e1;
         dc.eG[lane] = e0; dc.eG[lane + 32] = e1;
-        dc.eRest[lane] = ex2_approx(GC - G0); dc.eRest[lane + 32] = ex2_approx(GC - G1);
+        dc.bRest[lane] = b0 * (ex2_approx(GC - G0) * cinv); dc.bRest[lane + 32] = b1 * (ex2_approx(GC - G1) * cinv);
         const float G31 = __shfl_sync(0xffffffffu, G0, 31);
-        dc.colf[lane] = ex2_approx(G31 - G0);
-        if (lane == 0) { dc.eGC = ex2_approx(GC); dc.G2mid = G31; }
+        const float cf = ex2_approx(G31 - G0);
+        dc.colf[lane] = cf; dc.colfb[lane] = cf * b0;
+        if (lane == 0) { dc.wb = cprev * eGC; dc.G2mid = G31; dc.cfin = c; dc.rescale = rescale ? 1 : 0; }
         warp_arrive(cx.bar(B_DECAY_READY0 + (j & 3u)), lane);
     }
 }
@@ -521,15 +562,14 @@ __device__ __noinline__ uint32_t count_chunks(const TcParams& prm)
 }
 
 // ================================================================================================
-// warps 4-11: group G1.  Per iteration k: W^T epilogue of chunk k-1, Gram post-processing of chunk k+1
-// (writes A for the solve and the operand P), then T' and T'' of chunk k once group G2 has inverted it.
+// warps 4-11: group G1.  Per iteration k: Gram post-processing of chunk k+1 (writes A^ for the solve and the
+// operand P), then the W^T epilogue of chunk k.
 // ================================================================================================
 __device__ void role_g1(const Ctx& cx, const TcParams& prm, int wtid)
 {
     const int lane = wtid & 31, pw = wtid >> 5;          // pw = 0..7
     const int w4 = pw & 3, hf = pw >> 2;                 // TMEM lane window, column half
     const uint32_t tl = cx.tmem + ((uint32_t)(w4 * 32) << 16);
-    uint8_t* XH = cx.sm + SM_XH;
     Misc* misc = cx.misc;
     const uint32_t J = count_chunks(prm);
     GDN_TIMERS(long long tt_[16] = {0}; long long tl_ = clock64(); int nch = 0;)
@@ -542,7 +582,11 @@ __device__ void role_g1(const Ctx& cx, const TcParams& prm, int wtid)
         const int t = ((w4 & 1) << 5) + lane;
         const bool isA = w4 < 2;
         const float G2t = dc.G2[t];
-        const float rowscale = isA ? dc.beta[t] : 1.f;
+        // the solve works on A^ = strict_lower(Gam (K K^T)) diag(beta) (beta on the columns): its inverse P^ gives
+        // T' = diag(beta) P^ and T'' = diag(beta) P^ diag(e^G), and the common row factor beta moves into the
+        // Delta epilogue, so that P^ itself is one MMA operand and its column-scaled copy the other
+        const float* __restrict__ colscale = isA ? dc.beta : misc->ones;
+        const float* __restrict__ colfac = isA ? dc.colfb : dc.colf;
         const int t_lim = isA ? t : t + 1;                      // keep columns s < t_lim
         cx.wait(B_GRAM_DONE, c & 1u);
         tc_fence_after();
@@ -554,7 +598,7 @@ __device__ void role_g1(const Ctx& cx, const TcParams& prm, int wtid)
         // column blocks are dealt so that each warp of a lane window gets one block that touches the
         // diagonal and one that does not: half 0 -> blocks {0, 2}, half 1 -> blocks {1, 3}
         const bool lower_rows = (w4 & 1) != 0;                  // rows 32-63
-        const float rowf = lower_rows ? ex2_approx(G2t - dc.G2mid) * rowscale : 0.f;
+        const float rowf = lower_rows ? ex2_approx(G2t - dc.G2mid) : 0.f;
 #pragma unroll 1
         for (int g = 0; g < 2; ++g) {
             const int cb = hf + 2 * g, c0 = 16 * cb;
@@ -573,7 +617,7 @@ __device__ void role_g1(const Ctx& cx, const TcParams& prm, int wtid)
                 // every column precedes every row of this warp: Gam = rowf * colf, no mask, no exp
 #pragma unroll
                 for (int i4 = 0; i4 < 4; ++i4) {
-                    const float4 cf = *reinterpret_cast<const float4*>(&dc.colf[c0 + 4 * i4]);
+                    const float4 cf = *reinterpret_cast<const float4*>(&colfac[c0 + 4 * i4]);
                     vals[4 * i4 + 0] = (rowf * cf.x) * __uint_as_float(acc[4 * i4 + 0]);
                     vals[4 * i4 + 1] = (rowf * cf.y) * __uint_as_float(acc[4 * i4 + 1]);
                     vals[4 * i4 + 2] = (rowf * cf.z) * __uint_as_float(acc[4 * i4 + 2]);
@@ -583,12 +627,13 @@ __device__ void role_g1(const Ctx& cx, const TcParams& prm, int wtid)
 #pragma unroll
                 for (int i4 = 0; i4 < 4; ++i4) {
                     const float4 gs = *reinterpret_cast<const float4*>(&dc.G2[c0 + 4 * i4]);
-                    const float gss[4] = {gs.x, gs.y, gs.z, gs.w};
+                    const float4 cs = *reinterpret_cast<const float4*>(&colscale[c0 + 4 * i4]);
+                    const float gss[4] = {gs.x, gs.y, gs.z, gs.w}, css[4] = {cs.x, cs.y, cs.z, cs.w};
 #pragma unroll
                     for (int e = 0; e < 4; ++e) {
                         const int i = 4 * i4 + e;
                         // masked entries may overflow to inf / NaN before the select discards them
-                        const float f = ex2_approx(G2t - gss[e]) * rowscale;
+                        const float f = ex2_approx(G2t - gss[e]) * css[e];
                         vals[i] = (c0 + i < t_lim) ? f * __uint_as_float(acc[i]) : 0.f;
                     }
                 }
@@ -616,81 +661,27 @@ __device__ void role_g1(const Ctx& cx, const TcParams& prm, int wtid)
         warp_arrive(cx.bar(B_A_READY0 + (c & 1u)), lane);       // A of chunk c is complete: the solve may start
     };
 
-    // ---- T'' = X diag(beta e^G) (operand of the W^T MMA), T' = X diag(beta) (operand of the U^T MMA) ------
-    auto t_write = [&](uint32_t k) {
-        const Decay& dc = misc->decay[k & 3u];
-        cx.wait(B_X_READY, k & 1u);
-        // the T' buffer of chunk k was last read by the U^T MMA of chunk k-2; T'' by the W^T MMA of chunk k-1,
-        // whose completion the W^T epilogue of this iteration has already waited for
-        if (k >= 2) cx.wait(B_TP_FREE0 + (k & 1u), ((k >> 1) - 1u) & 1u);
-        const int tt = wtid >> 2, q = wtid & 3, c0 = 16 * q;   // row, 16-column quarter
-        float x[16];
-#pragma unroll
-        for (int c8 = 0; c8 < 2; ++c8) {
-            const uint4 xv = *reinterpret_cast<const uint4*>(XH + (tt * LDA + c0 + 8 * c8) * 2);
-            const uint32_t xw[4] = {xv.x, xv.y, xv.z, xv.w};
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-                const int s0 = c0 + 8 * c8 + 2 * e;
-                x[8 * c8 + 2 * e] = (s0 <= tt) ? bf_lo(xw[e]) : 0.f;
-                x[8 * c8 + 2 * e + 1] = (s0 + 1 <= tt) ? bf_hi(xw[e]) : 0.f;
-            }
-        }
-        warp_arrive(cx.bar(B_X_FREE), lane);                    // X has been read: the next solve may overwrite it
-        const uint32_t o0 = tt * 128 + (((2 * q) ^ (tt & 7)) << 4), o1 = tt * 128 + (((2 * q + 1) ^ (tt & 7)) << 4);
-        // T'' first: it is all the W^T MMA waits for, and that MMA then overlaps the T' half of this routine
-        {
-            uint32_t w2[8];
-#pragma unroll
-            for (int i4 = 0; i4 < 4; ++i4) {
-                const float4 ev = *reinterpret_cast<const float4*>(&dc.bE[c0 + 4 * i4]);
-                w2[2 * i4] = pack_bf16x2(x[4 * i4] * ev.x, x[4 * i4 + 1] * ev.y);
-                w2[2 * i4 + 1] = pack_bf16x2(x[4 * i4 + 2] * ev.z, x[4 * i4 + 3] * ev.w);
-            }
-            *reinterpret_cast<uint4*>(cx.sm + SM_TPP + o0) = make_uint4(w2[0], w2[1], w2[2], w2[3]);
-            *reinterpret_cast<uint4*>(cx.sm + SM_TPP + o1) = make_uint4(w2[4], w2[5], w2[6], w2[7]);
-            fence_proxy_async_smem();
-            warp_arrive(cx.bar(B_TPP_READY), lane);
-        }
-        {
-            uint32_t w1[8];
-#pragma unroll
-            for (int i4 = 0; i4 < 4; ++i4) {
-                const float4 bv = *reinterpret_cast<const float4*>(&dc.beta[c0 + 4 * i4]);
-                w1[2 * i4] = pack_bf16x2(x[4 * i4] * bv.x, x[4 * i4 + 1] * bv.y);
-                w1[2 * i4 + 1] = pack_bf16x2(x[4 * i4 + 2] * bv.z, x[4 * i4 + 3] * bv.w);
-            }
-            uint8_t* tp = cx.sm + SM_TP + (k & 1u) * 8192;
-            *reinterpret_cast<uint4*>(tp + o0) = make_uint4(w1[0], w1[1], w1[2], w1[3]);
-            *reinterpret_cast<uint4*>(tp + o1) = make_uint4(w1[4], w1[5], w1[6], w1[7]);
-            // made visible to the tensor core by the proxy fence of this chunk's W^T epilogue, which every
-            // thread executes before the arrival that releases the operand set
-        }
-    };
-
     // ---- W^T epilogue of chunk c: bf16 rows [dk][t] as the N-major operand of the S0 W^T MMA; completes the
-    // operand set of chunk c (each warp converts 32 columns of its lane window)
+    // operand set of chunk c (each warp converts 32 columns of its lane window; TMEM lane = key index)
     auto w_epilogue = [&](uint32_t c) {
-        cx.wait(B_W_DONE, c & 1u);
+        cx.wait(B_W_DONE0 + (c & 1u), (c >> 1) & 1u);
         tc_fence_after();
         // W^T is single-buffered: the S0 W^T MMA of chunk c-1 must have read it
         if (c >= 1) cx.wait(B_MMA1_DONE, (c - 1) & 1u);
-        const int drow = w4 * 32 + lane;                        // dk index = TMEM lane
+        const int drow = w4 * 32 + lane;
         uint8_t* wrow = cx.sm + SM_WT + drow * 128;
-        {
-            const int c0 = 32 * hf;
-            uint32_t acc[32];
-            tmem_ld32(tl + TM_WACC + c0, acc);
-            tmem_ld_wait();
+        const int c0 = 32 * hf;
+        uint32_t acc[32];
+        tmem_ld32(tl + TM_WACC + c0, acc);
+        tmem_ld_wait();
 #pragma unroll
-            for (int c8 = 0; c8 < 4; ++c8) {
-                uint4 u;
-                u.x = pack_bf16x2(__uint_as_float(acc[c8 * 8 + 0]), __uint_as_float(acc[c8 * 8 + 1]));
-                u.y = pack_bf16x2(__uint_as_float(acc[c8 * 8 + 2]), __uint_as_float(acc[c8 * 8 + 3]));
-                u.z = pack_bf16x2(__uint_as_float(acc[c8 * 8 + 4]), __uint_as_float(acc[c8 * 8 + 5]));
-                u.w = pack_bf16x2(__uint_as_float(acc[c8 * 8 + 6]), __uint_as_float(acc[c8 * 8 + 7]));
-                *reinterpret_cast<uint4*>(wrow + ((((c0 >> 3) + c8) ^ (drow & 7)) << 4)) = u;
-            }
+        for (int c8 = 0; c8 < 4; ++c8) {
+            uint4 u;
+            u.x = pack_bf16x2(__uint_as_float(acc[c8 * 8 + 0]), __uint_as_float(acc[c8 * 8 + 1]));
+            u.y = pack_bf16x2(__uint_as_float(acc[c8 * 8 + 2]), __uint_as_float(acc[c8 * 8 + 3]));
+            u.z = pack_bf16x2(__uint_as_float(acc[c8 * 8 + 4]), __uint_as_float(acc[c8 * 8 + 5]));
+            u.w = pack_bf16x2(__uint_as_float(acc[c8 * 8 + 6]), __uint_as_float(acc[c8 * 8 + 7]));
+            *reinterpret_cast<uint4*>(wrow + ((((c0 >> 3) + c8) ^ (drow & 7)) << 4)) = u;
         }
         tc_fence_before();
         warp_arrive(cx.bar(B_WACC_READ), lane);                 // the accumulator may take the next W^T tile
@@ -698,16 +689,14 @@ __device__ void role_g1(const Ctx& cx, const TcParams& prm, int wtid)
         warp_arrive(cx.bar(B_PRE_DONE0 + (c & 1u)), lane);
     };
 
-    if (J == 0) return;
-    // iteration i: W^T epilogue of chunk i-2 (first: it completes the operand set the chain is waiting for),
-    // Gram post-processing of chunk i (overlaps the solve of chunk i-1), T', T'' of chunk i-1
+    // iteration i: Gram post-processing of chunk i, then the W^T epilogue of chunk i-1, whose solve and W^T MMA
+    // ran meanwhile
 #pragma unroll 1
-    for (uint32_t i = 0; i <= J + 1; ++i) {
-        if (i >= 2) w_epilogue(i - 2);
+    for (uint32_t i = 0; i <= J; ++i) {
         GDN_T(0);
         if (i < J) post(i);
         GDN_T(1);
-        if (i >= 1 && i <= J) t_write(i - 1);
+        if (i >= 1) w_epilogue(i - 1);
         GDN_T(2);
         GDN_TIMERS(++nch;)
     }
@@ -721,19 +710,42 @@ __device__ void role_g1(const Ctx& cx, const TcParams& prm, int wtid)
 }
 
 // ================================================================================================
-// warps 20-21: group G2, X = (I + A)^-1 of chunk k while G1 works on its neighbours.  Each warp inverts one
-// 32 x 32 diagonal half without any cross-warp barrier:
+// warps 20-21: group G2, P^ = (I + A^)^-1 of chunk k.  Each warp inverts one 32 x 32 diagonal half without any
+// cross-warp barrier:
 //   level 0  : its four 8 x 8 diagonal blocks by forward substitution in fp32
 //   level 0.5: 8 -> 16 merges, level 1: the 16 -> 32 merge X[hi][lo] = -X[hi][hi] (A[hi][lo] X[lo][lo]),
 //   level 2  : X[32:64][0:32] = -X22 (A21 X11), two 16 x 16 tiles per warp,
-// the merges on mma.sync with ldmatrix-fed bf16 fragments.
+// the merges on mma.sync with ldmatrix-fed bf16 fragments.  The inverse is built in place in the T' operand
+// buffer (MMA operand layout, which ldmatrix reads just as well), and every block is also stored, with its
+// columns scaled by e^G, into the T'' operand buffer at the moment it is in registers; what lies above the
+// 16 x 16 diagonal blocks of both is zero from the start of the kernel.
 // ================================================================================================
+struct TOut {
+    uint8_t* tp; uint8_t* tpp; const float* eG;
+    __device__ __forceinline__ void pair(int row, int col, float v0, float v1) const       // col even
+    {
+        const uint32_t o = sw_off(row, col);
+        const float2 sc = *reinterpret_cast<const float2*>(eG + col);
+        *reinterpret_cast<uint32_t*>(tp + o) = pack_bf16x2(v0, v1);
+        *reinterpret_cast<uint32_t*>(tpp + o) = pack_bf16x2(v0 * sc.x, v1 * sc.y);
+    }
+    // sign * c of a 16 x 16 accumulator tile (two 8-column halves) at rows r0.., columns n0..
+    __device__ __forceinline__ void tile16(const float (&c)[2][4], float sign, int r0, int n0, int lane) const
+    {
+        const int g = lane >> 2, t4 = lane & 3;
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            pair(r0 + g, n0 + 8 * h + 2 * t4, sign * c[h][0], sign * c[h][1]);
+            pair(r0 + g + 8, n0 + 8 * h + 2 * t4, sign * c[h][2], sign * c[h][3]);
+        }
+    }
+};
+
 __device__ void role_g2(const Ctx& cx, const TcParams& prm, int wtid)
 {
     const int lane = wtid & 31, pw = wtid >> 5;          // pw = 0, 1
-    uint8_t* XH = cx.sm + SM_XH;
     uint8_t* MH = cx.sm + SM_MH;
-    const uint32_t xh = cx.sb + SM_XH, mh = cx.sb + SM_MH;
+    const uint32_t mh = cx.sb + SM_MH;
     const uint32_t J = count_chunks(prm);
     auto pair_sync = [&]() { asm volatile("bar.sync 3, 64;" ::: "memory"); };
     GDN_TIMERS(long long tt_[16] = {0}; long long tl_ = clock64(); int nch = 0;)
@@ -742,7 +754,14 @@ __device__ void role_g2(const Ctx& cx, const TcParams& prm, int wtid)
         const uint8_t* AH = cx.sm + SM_AH + (k & 1u) * AH_BYTES;
         const uint32_t ah = cx.sb + SM_AH + (k & 1u) * AH_BYTES;
         cx.wait(B_A_READY0 + (k & 1u), (k >> 1) & 1u);
-        if (k >= 1) cx.wait(B_X_FREE, (k - 1) & 1u);           // T', T'' of chunk k-1 have been formed from X
+        // operand buffers of chunk k: T' was last read by the U^T MMA of chunk k-2, T'' by the W^T MMA of chunk k-2
+        if (k >= 2) {
+            cx.wait(B_TP_FREE0 + (k & 1u), ((k >> 1) - 1u) & 1u);
+            cx.wait(B_W_DONE0 + (k & 1u), ((k >> 1) - 1u) & 1u);
+        }
+        const Decay& dc = cx.misc->decay[k & 3u];
+        const TOut to = {cx.sm + SM_TP + (k & 1u) * 8192, cx.sm + SM_TPP + (k & 1u) * 8192, dc.eG};
+        const uint32_t xs = cx.sb + SM_TP + (k & 1u) * 8192;     // the inverse under construction
         GDN_T(0);
         {
             const int bb = 4 * pw + (lane >> 3), b = 8 * bb, jj = lane & 7;
@@ -761,11 +780,13 @@ __device__ void role_g2(const Ctx& cx, const TcParams& prm, int wtid)
                 }
                 x[r] = (r > jj) ? -(acc0 + acc1) : x[r];
             }
-            const int zc = b + 8;                              // upper-right 8 x 8 of the 16 x 16 parent block
+            // this thread's column of the diagonal block, zeros above the diagonal included
+            const float sc = dc.eG[b + jj];
 #pragma unroll
             for (int r = 0; r < 8; ++r) {
-                *reinterpret_cast<__nv_bfloat16*>(XH + ((b + r) * LDA + b + jj) * 2) = __float2bfloat16_rn(x[r]);
-                if (!(bb & 1)) *reinterpret_cast<uint16_t*>(XH + ((b + r) * LDA + zc + jj) * 2) = 0;
+                const uint32_t o = sw_off(b + r, b + jj);
+                *reinterpret_cast<__nv_bfloat16*>(to.tp + o) = __float2bfloat16_rn(x[r]);
+                *reinterpret_cast<__nv_bfloat16*>(to.tpp + o) = __float2bfloat16_rn(x[r] * sc);
             }
         }
         __syncwarp();
@@ -774,7 +795,7 @@ __device__ void role_g2(const Ctx& cx, const TcParams& prm, int wtid)
             const int g = lane >> 2, t4 = lane & 3;
             uint32_t a[2], bx[2];
             ldm_x2(a, ah + ((b16 + 8 + rr) * LDA + b16) * 2);                    // A21 of both blocks
-            ldm_x2_trans(bx, xh + ((b16 + rr) * LDA + b16) * 2);                  // X11 of both blocks
+            ldm_x2_trans(bx, xs + sw_off(b16 + rr, b16));                         // X11 of both blocks
             float m0[4] = {0.f, 0.f, 0.f, 0.f}, m1[4] = {0.f, 0.f, 0.f, 0.f};
             mma_8x8(m0, a[0], bx[0]);
             mma_8x8(m1, a[1], bx[1]);
@@ -782,25 +803,25 @@ __device__ void role_g2(const Ctx& cx, const TcParams& prm, int wtid)
             *reinterpret_cast<uint32_t*>(MH + ((16 * pw + 8 + g) * LDM + 2 * t4) * 2) = pack_bf16x2(m1[0], m1[1]);
             __syncwarp();
             uint32_t a2[2], bm[2];
-            ldm_x2(a2, xh + ((b16 + 8 + rr) * LDA + b16 + 8) * 2);               // X22 of both blocks
+            ldm_x2(a2, xs + sw_off(b16 + 8 + rr, b16 + 8));                       // X22 of both blocks
             ldm_x2_trans(bm, mh + ((16 * pw + 8 * i + rr) * LDM) * 2);           // M of both blocks
             float d0[4] = {0.f, 0.f, 0.f, 0.f}, d1[4] = {0.f, 0.f, 0.f, 0.f};
             mma_8x8(d0, a2[0], bm[0]);
             mma_8x8(d1, a2[1], bm[1]);
             const int c0b = 32 * pw, c1b = 32 * pw + 16;
-            *reinterpret_cast<uint32_t*>(XH + ((c0b + 8 + g) * LDA + c0b + 2 * t4) * 2) = pack_bf16x2(-d0[0], -d0[1]);
-            *reinterpret_cast<uint32_t*>(XH + ((c1b + 8 + g) * LDA + c1b + 2 * t4) * 2) = pack_bf16x2(-d1[0], -d1[1]);
+            to.pair(c0b + 8 + g, c0b + 2 * t4, -d0[0], -d0[1]);
+            to.pair(c1b + 8 + g, c1b + 2 * t4, -d1[0], -d1[1]);
         }
         __syncwarp();
         {
             const int lo = 32 * pw, hi = 32 * pw + 16;
             float m[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
-            tile16_mma(m, ah, LDA, hi, lo, xh, LDA, lo, lo, lane);               // A[hi][lo] X[lo][lo]
+            tile16_mma_at(m, tile_addr(ah, LDA, hi, lo, lane), tile_addr_sw(xs, lo, lo, lane));       // A[hi][lo] X[lo][lo]
             tile16_store(m, 1.f, MH, LDM, 16 * pw, 0, lane);
             __syncwarp();
             float d[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
-            tile16_mma(d, xh, LDA, hi, hi, mh, LDM, 16 * pw, 0, lane);           // X[hi][hi] M
-            tile16_store(d, -1.f, XH, LDA, hi, lo, lane);
+            tile16_mma_at(d, tile_addr_sw(xs, hi, hi, lane), tile_addr(mh, LDM, 16 * pw, 0, lane));   // X[hi][hi] M
+            to.tile16(d, -1.f, hi, lo, lane);
         }
         pair_sync();
         GDN_T(1);
@@ -810,25 +831,28 @@ __device__ void role_g2(const Ctx& cx, const TcParams& prm, int wtid)
             const int mt = pw;
             float m0[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}}, m1[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
             // X11 is lower triangular: block column nt starts at block row nt
-            tile16_mma(m0, ah, LDA, 32 + 16 * mt, 0, xh, LDA, 0, 0, lane);
-            tile16_mma(m1, ah, LDA, 32 + 16 * mt, 16, xh, LDA, 16, 16, lane);
-            tile16_mma(m0, ah, LDA, 32 + 16 * mt, 16, xh, LDA, 16, 0, lane);
+            tile16_mma_at(m0, tile_addr(ah, LDA, 32 + 16 * mt, 0, lane), tile_addr_sw(xs, 0, 0, lane));
+            tile16_mma_at(m1, tile_addr(ah, LDA, 32 + 16 * mt, 16, lane), tile_addr_sw(xs, 16, 16, lane));
+            tile16_mma_at(m0, tile_addr(ah, LDA, 32 + 16 * mt, 16, lane), tile_addr_sw(xs, 16, 0, lane));
             tile16_store(m0, 1.f, MH, LDM, 16 * mt, 0, lane);
             tile16_store(m1, 1.f, MH, LDM, 16 * mt, 16, lane);
             warp_arrive(cx.bar(B_A_FREE0 + (k & 1u)), lane);   // last read of this chunk's A
             pair_sync();
             float d0[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}}, d1[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
             // X22 is lower triangular: block row mt ends at block column mt
-            tile16_mma(d0, xh, LDA, 32 + 16 * mt, 32, mh, LDM, 0, 0, lane);
-            tile16_mma(d1, xh, LDA, 32 + 16 * mt, 32, mh, LDM, 0, 16, lane);
+            tile16_mma_at(d0, tile_addr_sw(xs, 32 + 16 * mt, 32, lane), tile_addr(mh, LDM, 0, 0, lane));
+            tile16_mma_at(d1, tile_addr_sw(xs, 32 + 16 * mt, 32, lane), tile_addr(mh, LDM, 0, 16, lane));
             if (mt == 1) {
-                tile16_mma(d0, xh, LDA, 48, 48, mh, LDM, 16, 0, lane);
-                tile16_mma(d1, xh, LDA, 48, 48, mh, LDM, 16, 16, lane);
+                tile16_mma_at(d0, tile_addr_sw(xs, 48, 48, lane), tile_addr(mh, LDM, 16, 0, lane));
+                tile16_mma_at(d1, tile_addr_sw(xs, 48, 48, lane), tile_addr(mh, LDM, 16, 16, lane));
             }
-            tile16_store(d0, -1.f, XH, LDA, 32 + 16 * mt, 0, lane);
-            tile16_store(d1, -1.f, XH, LDA, 32 + 16 * mt, 16, lane);
+            to.tile16(d0, -1.f, 32 + 16 * mt, 0, lane);
+            to.tile16(d1, -1.f, 32 + 16 * mt, 16, lane);
         }
-        warp_arrive(cx.bar(B_X_READY), lane);
+        fence_proxy_async_smem();                               // T' and T'' are MMA operands
+        warp_arrive(cx.bar(B_TPP_READY), lane);
+        warp_arrive(cx.bar(B_TP_READY0 + (k & 1u)), lane);
+        pair_sync();                                            // the merge scratch is free for the next chunk
         GDN_T(2);
         GDN_TIMERS(++nch;)
     }
@@ -854,7 +878,9 @@ __device__ void role_chain(const Ctx& cx, const TcParams& prm, int wtid)
     Misc* misc = cx.misc;
     __nv_bfloat16* __restrict__ og = reinterpret_cast<__nv_bfloat16*>(p.out_o);
     const uint32_t num_items = (uint32_t)p.num_seqs * (uint32_t)p.Hv;
+    const uint32_t J = count_chunks(prm);
     GDN_TIMERS(long long tt_[16] = {0}; long long tl_ = clock64(); int nch = 0;)
+
 
     uint32_t j = 0;
 #pragma unroll 1
@@ -879,7 +905,7 @@ __device__ void role_chain(const Ctx& cx, const TcParams& prm, int wtid)
             GDN_DBG(const bool dbg = prm.debug && blockIdx.x == 0 && r == 0 && c < 2; float* dbase = prm.debug + c * DBG_STRIDE;)
 
             // ---- Delta epilogue: bf16 Delta^T and decayed Delta'^T as TMEM A operands ----------------------
-            cx.wait(B_PRE_DONE0 + (j & 1u), (j >> 1) & 1u);      // decay factors of this chunk are published
+            cx.wait(B_DECAY_READY0 + (j & 3u), (j >> 2) & 1u);   // decay factors of this chunk are published
             GDN_T(0);
             cx.wait(B_MMA1_DONE, j & 1u);
             GDN_T(1);
@@ -898,11 +924,13 @@ __device__ void role_chain(const Ctx& cx, const TcParams& prm, int wtid)
 #endif
 #pragma unroll
                 for (int i4 = 0; i4 < 4; ++i4) {
-                    const float4 er = *reinterpret_cast<const float4*>(&dc.eRest[c0 + 4 * i4]);
+                    // the accumulator holds Delta~^T = Delta^T diag(beta)^-1 (see the Gram post-processing)
+                    const float4 bt = *reinterpret_cast<const float4*>(&dc.beta[c0 + 4 * i4]);
+                    const float4 er = *reinterpret_cast<const float4*>(&dc.bRest[c0 + 4 * i4]);
                     const float a0 = __uint_as_float(acc[4 * i4]), a1 = __uint_as_float(acc[4 * i4 + 1]);
                     const float a2 = __uint_as_float(acc[4 * i4 + 2]), a3 = __uint_as_float(acc[4 * i4 + 3]);
-                    d1[2 * i4] = pack_bf16x2(a0, a1);
-                    d1[2 * i4 + 1] = pack_bf16x2(a2, a3);
+                    d1[2 * i4] = pack_bf16x2(a0 * bt.x, a1 * bt.y);
+                    d1[2 * i4 + 1] = pack_bf16x2(a2 * bt.z, a3 * bt.w);
                     d2[2 * i4] = pack_bf16x2(a0 * er.x, a1 * er.y);
                     d2[2 * i4 + 1] = pack_bf16x2(a2 * er.z, a3 * er.w);
                 }
@@ -914,13 +942,16 @@ __device__ void role_chain(const Ctx& cx, const TcParams& prm, int wtid)
             warp_arrive(cx.bar(B_D_READY), lane);
             GDN_T(2);
 
-            // ---- state: bf16 copy for the next chunk's MMAs + pre-scaling, or the final state ----------------
-            // total decay of the next chunk scales the carried state ahead of that chunk's update MMA
-            float eGCnext = 1.f;
+            // ---- state: bf16 copy for the next chunk's MMAs, or the final state ------------------------------
+            // if the next chunk starts from a rescaled state, the stored state is multiplied by wb on the way
+            float wb = 1.f;
+            bool rescale = false;
             if (!last) {
                 cx.wait(B_DECAY_READY0 + ((j + 1) & 3u), ((j + 1) >> 2) & 1u);
-                eGCnext = misc->decay[(j + 1) & 3u].eGC;
+                wb = misc->decay[(j + 1) & 3u].wb;
+                rescale = misc->decay[(j + 1) & 3u].rescale != 0;
             }
+            const float cfin = dc.cfin;
             cx.wait(B_MMA3_DONE, j & 1u);
             GDN_T(3);
             tc_fence_after();
@@ -942,11 +973,13 @@ __device__ void role_chain(const Ctx& cx, const TcParams& prm, int wtid)
                     uint32_t pk[8];
 #pragma unroll
                     for (int i = 0; i < 8; ++i) pk[i] = pack_bf16x2(__uint_as_float(acc[2 * i]), __uint_as_float(acc[2 * i + 1]));
-#pragma unroll
-                    for (int i = 0; i < 16; ++i) acc[i] = __float_as_uint(__uint_as_float(acc[i]) * eGCnext);
                     GDN_DBG(long long s2_ = clock64();)
                     tmem_st8(tl + TM_SBF + (c0 >> 1), pk);
-                    tmem_st16(tl + TM_S32 + c0, acc);
+                    if (rescale) {
+#pragma unroll
+                        for (int i = 0; i < 16; ++i) acc[i] = __float_as_uint(__uint_as_float(acc[i]) * wb);
+                        tmem_st16(tl + TM_S32 + c0, acc);
+                    }
                     GDN_DBG(long long s3_ = clock64();
                             if (prm.debug && blockIdx.x == 0 && wtid == 0 && j == 10) {
                                 float* d = prm.debug + 2 * DBG_STRIDE + 32 + g * 4;
@@ -954,7 +987,7 @@ __device__ void role_chain(const Ctx& cx, const TcParams& prm, int wtid)
                             })
                 } else if (st_out) {
 #pragma unroll
-                    for (int i = 0; i < 16; ++i) st_out[(c0 + i) * 128 + dv] = __uint_as_float(acc[i]);
+                    for (int i = 0; i < 16; ++i) st_out[(c0 + i) * 128 + dv] = __uint_as_float(acc[i]) * cfin;
                 }
             }
             tmem_st_wait();
@@ -1053,11 +1086,12 @@ gdn_tc_kernel(const TcParams prm, const __grid_constant__ CUtensorMap tm_q,
     if (tid == 32) {
         for (int i = 0; i < NUM_BARS; ++i) {
             // arrivals per phase: one per warp of the arriving group (G1 and chain: 8 warps, G2: 2 warps)
-            const bool wg_bar = i == B_GRAM_READ || i == B_TPP_READY || i == B_D_READY || i == B_SBF_READY ||
+            const bool wg_bar = i == B_GRAM_READ || i == B_D_READY || i == B_SBF_READY ||
                                 i == B_WACC_READ || i == B_PRE_DONE0 || i == B_PRE_DONE1 ||
-                                i == B_A_READY0 || i == B_A_READY1 || i == B_X_FREE;
+                                i == B_A_READY0 || i == B_A_READY1;
             const bool out_bar = i == B_ACC23_FREE || (i >= B_DECAY_FREE0 && i <= B_DECAY_FREE3);
-            const bool g2_bar = i == B_A_FREE0 || i == B_A_FREE1 || i == B_X_READY;
+            const bool g2_bar = i == B_A_FREE0 || i == B_A_FREE1 || i == B_TPP_READY || i == B_TP_READY0 ||
+                                i == B_TP_READY1;
             mbar_init(cx.bar(i), wg_bar ? 8u : out_bar ? 4u : g2_bar ? 2u : 1u);
         }
         fence_mbar_init();
@@ -1065,6 +1099,12 @@ gdn_tc_kernel(const TcParams prm, const __grid_constant__ CUtensorMap tm_q,
         cx.misc->timeout_ns = prm.wait_timeout_ns;
         prefetch_tmap(&tm_q); prefetch_tmap(&tm_k); prefetch_tmap(&tm_v);
     }
+    // the operand tiles T', T'' (two buffers each, contiguous) are only ever written on and below their 16 x 16
+    // diagonal blocks: everything else is zeroed once, here
+    for (uint32_t i = tid; i < 4u * 8192u / 16u; i += kThreads)
+        *reinterpret_cast<uint4*>(cx.sm + SM_TP + i * 16u) = make_uint4(0u, 0u, 0u, 0u);
+    if (tid < 64) cx.misc->ones[tid] = 1.f;
+    fence_proxy_async_smem();
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -1093,8 +1133,9 @@ gdn_tc_kernel(const TcParams prm, const __grid_constant__ CUtensorMap tm_q,
         role_out(cx, prm, warp, lane);
     }
 #ifdef GDN_TC_PROFILE
-    if (prm.debug && blockIdx.x == 0 && lane == 0 && (warp < 3 || warp == 4 || warp == 12 || warp == 20)) {
-        const int slot = warp < 3 ? warp : (warp == 4 ? 3 : (warp == 12 ? 4 : 8));
+    if (prm.debug && blockIdx.x == 0 && lane == 0 &&
+        (warp <= 4 || warp == 12 || warp == 20 || warp == 22 || warp == 23)) {
+        const int slot = warp < 3 ? warp : (warp == 4 ? 3 : (warp == 12 ? 4 : (warp == 20 ? 8 : (warp == 22 ? 9 : (warp == 23 ? 10 : 11)))));
         cx.prof_dump(prm.debug + slot * 48);
     }
 #endif
