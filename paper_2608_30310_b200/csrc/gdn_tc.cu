@@ -70,7 +70,7 @@ constexpr uint32_t SM_MISC = ((SM_MH + 32 * LDM * 2 + 1023) / 1024) * 1024;
 
 enum Bar {
     B_FULL_KQ0 = 0, B_FULL_KQ1, B_FULL_KQ2, B_FULL_V, B_GRAM_DONE, B_W_DONE0, B_W_DONE1, B_U_DONE, B_MMA1_DONE,
-    B_MMA3_DONE, B_KQ_FREE0, B_KQ_FREE1, B_KQ_FREE2, B_P_FREE0, B_P_FREE1, B_P_FREE2, B_TP_FREE0, B_TP_FREE1,
+    B_MMA3_DONE, B_STATE_DONE, B_KQ_FREE0, B_KQ_FREE1, B_KQ_FREE2, B_P_FREE0, B_P_FREE1, B_P_FREE2, B_TP_FREE0, B_TP_FREE1,
     B_GRAM_READ, B_WACC_READ, B_TPP_READY,
     B_PRE_DONE0, B_PRE_DONE1, B_D_READY, B_SBF_READY, B_ACC23_FREE,
     B_DECAY_READY0, B_DECAY_READY1, B_DECAY_READY2, B_DECAY_READY3,
@@ -110,11 +110,10 @@ constexpr uint32_t TM_ACC2 = 256;   // S0 Q^T, 64 columns
 constexpr uint32_t TM_ACC3 = 320;   // Delta^T P^T, 64 columns
 constexpr uint32_t TM_GRAM = 384;   // Gram accumulator, 64 columns
 constexpr uint32_t TM_WACC = 448;   // W^T accumulator, 64 columns
-// The bf16 Delta operands reuse the columns of the bf16 state copy: the copy is dead once the MMAs that read
-// it have completed (which the Delta epilogue waits for), and it is rewritten only after the MMAs that read
-// the Delta operands have completed.
-constexpr uint32_t TM_DBF = 128;    // Delta^T bf16, 32 columns
-constexpr uint32_t TM_DPBF = 160;   // (Delta diag(e^{G_C - G}))^T bf16, 32 columns
+// The bf16 A operands Delta^T and Delta'^T replace the fp32 accumulator they are computed from, in place: the 16
+// fp32 columns of tokens [16 s, 16 s + 16) become 8 columns of Delta^T followed by 8 columns of Delta'^T.
+constexpr uint32_t TM_DBF = TM_ACC1;        // + 16 s
+constexpr uint32_t TM_DPBF = TM_ACC1 + 8;   // + 16 s
 
 constexpr uint32_t ID_GRAM = idesc_bf16(128, 64, 0, 0, 0);    // [K;Q] (K-major) x K (K-major)
 constexpr uint32_t ID_WU = idesc_bf16(128, 64, 1, 0, 0);      // K^T or V^T (M-major) x T (K-major)
@@ -473,30 +472,32 @@ __device__ void role_mma_chain(const Ctx& cx, const TcParams& prm)
                 mma_ts(cx.tmem + TM_ACC1, cx.tmem + TM_SBF + ks * 8, desc_add(d_wt, ks * 2048), ID_SW, 1u);
         }
         __syncwarp();
+        // Delta^T is complete: its epilogue starts now
+        if (elect_one()) mma_commit(cx.bar(B_MMA1_DONE));
+        __syncwarp();
+        cx.wait(B_D_READY, j & 1u);
+        // the two output accumulators were read by the output epilogue of chunk j-1, a whole Delta epilogue ago
         if (j >= 1) cx.wait(B_ACC23_FREE, (j - 1) & 1u);
         tc_fence_after();
         if (elect_one()) {
+            // S0 Q^T before the state update: the state epilogue overwrites the bf16 state as soon as that update
+            // is complete, and completion is in issue order
             if (!first) {
 #pragma unroll
                 for (int ks = 0; ks < 8; ++ks)
                     mma_ts(cx.tmem + TM_ACC2, cx.tmem + TM_SBF + ks * 8,
                            desc_add(d_q, (ks >> 2) * 16384 + (ks & 3) * 32), ID_SQ, ks > 0);
             }
-            mma_commit(cx.bar(B_MMA1_DONE));
-        }
-        __syncwarp();
-        cx.wait(B_D_READY, j & 1u);
-        tc_fence_after();
-        if (elect_one()) {
 #pragma unroll
             for (int ks = 0; ks < 4; ++ks)
-                mma_ts(cx.tmem + TM_ACC3, cx.tmem + TM_DBF + ks * 8, desc_add(d_p, ks * 32), ID_DP, ks > 0);
-#pragma unroll
-            for (int ks = 0; ks < 4; ++ks)
-                mma_ts(cx.tmem + TM_S32, cx.tmem + TM_DPBF + ks * 8, desc_add(d_kn, ks * 2048), ID_DK,
+                mma_ts(cx.tmem + TM_S32, cx.tmem + TM_DPBF + ks * 16, desc_add(d_kn, ks * 2048), ID_DK,
                        (!first || ks > 0) ? 1u : 0u);
+            mma_commit(cx.bar(B_STATE_DONE));
+            mma_commit(cx.bar(B_KQ_FREE0 + j % 3u));            // K and Q of this chunk have been read
+#pragma unroll
+            for (int ks = 0; ks < 4; ++ks)
+                mma_ts(cx.tmem + TM_ACC3, cx.tmem + TM_DBF + ks * 16, desc_add(d_p, ks * 32), ID_DP, ks > 0);
             mma_commit(cx.bar(B_MMA3_DONE));
-            mma_commit(cx.bar(B_KQ_FREE0 + j % 3u));
             mma_commit(cx.bar(B_P_FREE0 + j % 3u));
         }
         __syncwarp();
@@ -934,8 +935,8 @@ __device__ void role_chain(const Ctx& cx, const TcParams& prm, int wtid)
                     d2[2 * i4] = pack_bf16x2(a0 * er.x, a1 * er.y);
                     d2[2 * i4 + 1] = pack_bf16x2(a2 * er.z, a3 * er.w);
                 }
-                tmem_st8(tl + TM_DBF + (c0 >> 1), d1);
-                tmem_st8(tl + TM_DPBF + (c0 >> 1), d2);
+                tmem_st8(tl + TM_DBF + c0, d1);
+                tmem_st8(tl + TM_DPBF + c0, d2);
             }
             tmem_st_wait();
             tc_fence_before();
@@ -952,7 +953,7 @@ __device__ void role_chain(const Ctx& cx, const TcParams& prm, int wtid)
                 rescale = misc->decay[(j + 1) & 3u].rescale != 0;
             }
             const float cfin = dc.cfin;
-            cx.wait(B_MMA3_DONE, j & 1u);
+            cx.wait(B_STATE_DONE, j & 1u);
             GDN_T(3);
             tc_fence_after();
 #pragma unroll 1
