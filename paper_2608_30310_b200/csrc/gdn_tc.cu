@@ -20,7 +20,7 @@
 //                                              c the running product of the chunk decays, folded into the
 //                                              per-token factors; rescaled before c drops below 2^-40)
 //
-// The CTA is warp-specialised and software-pipelined over the chunks of all chains it owns (27 warps):
+// The CTA is warp-specialised and software-pipelined over the chunks of all chains it owns (28 warps):
 //   warp 0       TMA producer: K/Q tiles two chunks ahead (3 slots), V one chunk ahead (1 slot)
 //   warp 1       issues the chain MMAs (U^T, S0 W^T, S0 Q^T, Dl^T P^T, state update)
 //   warp 2       issues the Gram MMAs, two chunks ahead of the chain
@@ -29,10 +29,10 @@
 //   warps 4-11   group G1 (two warps per TMEM lane window): Gram post-processing (A^, P) of chunk k+1, then the
 //                W^T epilogue of chunk k
 //   warps 12-19  chain group: Delta epilogue, state conversion (and rescaling when due), final state (chunk j)
-//   warps 20-21  group G2: the triangular solve of chunk k, built in place in the T' operand buffer, with the
-//                column-scaled copy written to the T'' operand buffer block by block
-//   warp 22      issues the W^T MMAs
-//   warps 23-26  output group: output epilogue of chunk j, off the chain's critical path
+//   warps 20-23  group G2, two teams of two warps that take alternate chunks: the triangular solve, built in
+//                place in the T' operand buffer, with the column-scaled copy written to the T'' operand buffer
+//                block by block; the team then issues the W^T MMA itself
+//   warps 24-27  output group: output epilogue of chunk j, off the chain's critical path
 // Every per-chunk loop is kept rolled with 16-column TMEM accesses: straight-line code larger than the
 // instruction caches runs at a fraction of the issue rate, so the static footprint matters as much as the
 // instruction count.
@@ -52,7 +52,7 @@ using namespace ptx;
 constexpr int LDA = 72;                       // bf16 row stride of the A and X scratch (144 B: conflict-free ldmatrix)
 constexpr int LDM = 40;                       // bf16 row stride of the merge scratch (80 B)
 constexpr float kLog2e = 1.4426950408889634f;
-constexpr int kThreads = 864;      // 27 warps, see the role table above
+constexpr int kThreads = 896;      // 28 warps, see the role table above (at most 72 registers per thread)
 constexpr int kWgThreads = 256;
 
 // ---- shared memory map (bytes from a 1024-aligned base) ---------------------------------------
@@ -66,12 +66,13 @@ constexpr uint32_t SM_P = 163840;             // 3 x P [t][s] bf16              
 constexpr uint32_t SM_AH = 188416;            // 2 x A bf16 [64][LDA]
 constexpr uint32_t AH_BYTES = 64 * LDA * 2;
 constexpr uint32_t SM_MH = SM_AH + 2 * AH_BYTES;   // merge scratch of the solve, bf16 [32][LDM]
-constexpr uint32_t SM_MISC = ((SM_MH + 32 * LDM * 2 + 1023) / 1024) * 1024;
+constexpr uint32_t MH_BYTES = 32 * LDM * 2;        // one per solve team
+constexpr uint32_t SM_MISC = ((SM_MH + 2 * MH_BYTES + 1023) / 1024) * 1024;
 
 enum Bar {
     B_FULL_KQ0 = 0, B_FULL_KQ1, B_FULL_KQ2, B_FULL_V, B_GRAM_DONE, B_W_DONE0, B_W_DONE1, B_U_DONE, B_MMA1_DONE,
     B_MMA3_DONE, B_STATE_DONE, B_KQ_FREE0, B_KQ_FREE1, B_KQ_FREE2, B_P_FREE0, B_P_FREE1, B_P_FREE2, B_TP_FREE0, B_TP_FREE1,
-    B_GRAM_READ, B_WACC_READ, B_TPP_READY,
+    B_GRAM_READ, B_WACC_READ,
     B_PRE_DONE0, B_PRE_DONE1, B_D_READY, B_SBF_READY, B_ACC23_FREE,
     B_DECAY_READY0, B_DECAY_READY1, B_DECAY_READY2, B_DECAY_READY3,
     B_DECAY_FREE0, B_DECAY_FREE1, B_DECAY_FREE2, B_DECAY_FREE3,
@@ -410,30 +411,6 @@ __device__ void role_mma_gram(const Ctx& cx, const TcParams& prm)
 }
 
 // ================================================================================================
-// warp 22: W^T MMAs.  W^T(j) = K^T T''^T needs T''(j) and the accumulator read by chunk j-1.
-// ================================================================================================
-__device__ void role_mma_w(const Ctx& cx, const TcParams& prm)
-{
-    ChunkCursor cc;
-    cc.init(&prm.p, prm.s.order);
-#pragma unroll 1
-    for (uint32_t j = 0; cc.valid; ++j, cc.advance()) {
-        const uint64_t d_kt = smem_desc_sw128(cx.sb + SM_KQ + (j % 3u) * KQ_SLOT, 16384, 1024);   // K^T, M-major
-        const uint64_t d_tpp = smem_desc_sw128(cx.sb + SM_TPP + (j & 1u) * 8192, 16, 1024);
-        cx.wait(B_TPP_READY, j & 1u);
-        if (j >= 1) cx.wait(B_WACC_READ, (j - 1) & 1u);
-        tc_fence_after();
-        if (elect_one()) {
-#pragma unroll
-            for (int ks = 0; ks < 4; ++ks)
-                mma_ss(cx.tmem + TM_WACC, desc_add(d_kt, ks * 2048), desc_add(d_tpp, ks * 32), ID_WU, ks > 0);
-            mma_commit(cx.bar(B_W_DONE0 + (j & 1u)));
-        }
-        __syncwarp();
-    }
-}
-
-// ================================================================================================
 // warp 1: chain MMAs
 // ================================================================================================
 __device__ void role_mma_chain(const Ctx& cx, const TcParams& prm)
@@ -711,7 +688,8 @@ __device__ void role_g1(const Ctx& cx, const TcParams& prm, int wtid)
 }
 
 // ================================================================================================
-// warps 20-21: group G2, P^ = (I + A^)^-1 of chunk k.  Each warp inverts one 32 x 32 diagonal half without any
+// warps 20-23: group G2 (two teams of two warps on alternate chunks), P^ = (I + A^)^-1 of chunk k.  Each warp of a
+// team inverts one 32 x 32 diagonal half without any
 // cross-warp barrier:
 //   level 0  : its four 8 x 8 diagonal blocks by forward substitution in fp32
 //   level 0.5: 8 -> 16 merges, level 1: the 16 -> 32 merge X[hi][lo] = -X[hi][hi] (A[hi][lo] X[lo][lo]),
@@ -742,16 +720,17 @@ struct TOut {
     }
 };
 
-__device__ void role_g2(const Ctx& cx, const TcParams& prm, int wtid)
+__device__ void role_g2(const Ctx& cx, const TcParams& prm, int wtid, int team)
 {
     const int lane = wtid & 31, pw = wtid >> 5;          // pw = 0, 1
-    uint8_t* MH = cx.sm + SM_MH;
-    const uint32_t mh = cx.sb + SM_MH;
+    uint8_t* MH = cx.sm + SM_MH + team * MH_BYTES;
+    const uint32_t mh = cx.sb + SM_MH + team * MH_BYTES;
     const uint32_t J = count_chunks(prm);
-    auto pair_sync = [&]() { asm volatile("bar.sync 3, 64;" ::: "memory"); };
+    auto pair_sync = [&]() { asm volatile("bar.sync %0, 64;" ::"r"(3 + team) : "memory"); };
     GDN_TIMERS(long long tt_[16] = {0}; long long tl_ = clock64(); int nch = 0;)
+    // team 0 takes the even chunks, team 1 the odd ones: the A, T' and T'' buffers alternate the same way
 #pragma unroll 1
-    for (uint32_t k = 0; k < J; ++k) {
+    for (uint32_t k = (uint32_t)team; k < J; k += 2) {
         const uint8_t* AH = cx.sm + SM_AH + (k & 1u) * AH_BYTES;
         const uint32_t ah = cx.sb + SM_AH + (k & 1u) * AH_BYTES;
         cx.wait(B_A_READY0 + (k & 1u), (k >> 1) & 1u);
@@ -851,9 +830,22 @@ __device__ void role_g2(const Ctx& cx, const TcParams& prm, int wtid)
             to.tile16(d1, -1.f, 32 + 16 * mt, 16, lane);
         }
         fence_proxy_async_smem();                               // T' and T'' are MMA operands
-        warp_arrive(cx.bar(B_TPP_READY), lane);
         warp_arrive(cx.bar(B_TP_READY0 + (k & 1u)), lane);
-        pair_sync();                                            // the merge scratch is free for the next chunk
+        pair_sync();                                            // both warps' parts of T'' are in place
+        // W~^T = K^T T''^T, issued from here: needs the accumulator read by the W^T epilogue of chunk k-1
+        if (pw == 0) {
+            const uint64_t d_kt = smem_desc_sw128(cx.sb + SM_KQ + (k % 3u) * KQ_SLOT, 16384, 1024);   // K^T, M-major
+            const uint64_t d_tpp = smem_desc_sw128(cx.sb + SM_TPP + (k & 1u) * 8192, 16, 1024);
+            if (k >= 1) cx.wait(B_WACC_READ, (k - 1) & 1u);
+            tc_fence_after();
+            if (elect_one()) {
+#pragma unroll
+                for (int ks = 0; ks < 4; ++ks)
+                    mma_ss(cx.tmem + TM_WACC, desc_add(d_kt, ks * 2048), desc_add(d_tpp, ks * 32), ID_WU, ks > 0);
+                mma_commit(cx.bar(B_W_DONE0 + (k & 1u)));
+            }
+            __syncwarp();
+        }
         GDN_T(2);
         GDN_TIMERS(++nch;)
     }
@@ -1016,7 +1008,7 @@ __device__ void role_chain(const Ctx& cx, const TcParams& prm, int wtid)
 }
 
 // ================================================================================================
-// warps 23-26: output group (one warp per TMEM lane window).  O^T = diag(e^G) (S0 Q^T) + Delta^T P^T of chunk j,
+// warps 24-27: output group (one warp per TMEM lane window).  O^T = diag(e^G) (S0 Q^T) + Delta^T P^T of chunk j,
 // read from the two accumulators as soon as the chunk's last MMAs have completed and stored off the chain's
 // critical path.  For a fixed token the 128 lanes hold 128 consecutive bf16 of out_o: each warp store writes
 // 64 contiguous bytes (two full sectors), so the outputs go straight from registers to global memory.
@@ -1091,8 +1083,7 @@ gdn_tc_kernel(const TcParams prm, const __grid_constant__ CUtensorMap tm_q,
                                 i == B_WACC_READ || i == B_PRE_DONE0 || i == B_PRE_DONE1 ||
                                 i == B_A_READY0 || i == B_A_READY1;
             const bool out_bar = i == B_ACC23_FREE || (i >= B_DECAY_FREE0 && i <= B_DECAY_FREE3);
-            const bool g2_bar = i == B_A_FREE0 || i == B_A_FREE1 || i == B_TPP_READY || i == B_TP_READY0 ||
-                                i == B_TP_READY1;
+            const bool g2_bar = i == B_A_FREE0 || i == B_A_FREE1 || i == B_TP_READY0 || i == B_TP_READY1;
             mbar_init(cx.bar(i), wg_bar ? 8u : out_bar ? 4u : g2_bar ? 2u : 1u);
         }
         fence_mbar_init();
@@ -1126,17 +1117,15 @@ gdn_tc_kernel(const TcParams prm, const __grid_constant__ CUtensorMap tm_q,
         role_g1(cx, prm, tid - 128);
     } else if (warp >= 12 && warp < 20) {
         role_chain(cx, prm, tid - 384);
-    } else if (warp >= 20 && warp < 22) {
-        role_g2(cx, prm, tid - 640);
-    } else if (warp == 22) {
-        role_mma_w(cx, prm);
-    } else if (warp >= 23) {
+    } else if (warp >= 20 && warp < 24) {
+        role_g2(cx, prm, (tid - 640) & 63, (warp - 20) >> 1);
+    } else if (warp >= 24) {
         role_out(cx, prm, warp, lane);
     }
 #ifdef GDN_TC_PROFILE
     if (prm.debug && blockIdx.x == 0 && lane == 0 &&
-        (warp <= 4 || warp == 12 || warp == 20 || warp == 22 || warp == 23)) {
-        const int slot = warp < 3 ? warp : (warp == 4 ? 3 : (warp == 12 ? 4 : (warp == 20 ? 8 : (warp == 22 ? 9 : (warp == 23 ? 10 : 11)))));
+        (warp <= 4 || warp == 12 || warp == 20 || warp == 24)) {
+        const int slot = warp < 3 ? warp : (warp == 4 ? 3 : (warp == 12 ? 4 : (warp == 20 ? 8 : (warp == 24 ? 10 : 11))));
         cx.prof_dump(prm.debug + slot * 48);
     }
 #endif
