@@ -427,11 +427,11 @@ __device__ void role_mma_chain(const Ctx& cx, const TcParams& prm)
         const uint64_t d_p = smem_desc_sw128(cx.sb + SM_P + (j % 3u) * 8192, 16, 1024);
         const uint64_t d_tp = smem_desc_sw128(cx.sb + SM_TP + (j & 1u) * 8192, 16, 1024);
         const bool first = cc.first();
-        cx.wait(B_PRE_DONE0 + (j & 1u), (j >> 1) & 1u);
         cx.wait(B_TP_READY0 + (j & 1u), (j >> 1) & 1u);
         cx.wait(B_FULL_V, j & 1u);
         tc_fence_after();
-        // U^T = V^T T'^T -> ACC1 (free: the Delta epilogue of chunk j-1 came before that chunk's last MMAs)
+        // U^T = V^T T'^T -> ACC1 (free: the Delta operands of chunk j-1 in it were read by MMAs issued before
+        // these).  Issued ahead of the wait for the W^T operand, which is the last piece of the set to arrive.
         if (elect_one()) {
 #pragma unroll
             for (int ks = 0; ks < 4; ++ks)
@@ -440,6 +440,7 @@ __device__ void role_mma_chain(const Ctx& cx, const TcParams& prm)
             mma_commit(cx.bar(B_TP_FREE0 + (j & 1u)));
         }
         __syncwarp();
+        cx.wait(B_PRE_DONE0 + (j & 1u), (j >> 1) & 1u);
         // state of the previous chunk converted (or, at a chain start, the previous chain's state read out)
         if (j >= 1) cx.wait(B_SBF_READY, (j - 1) & 1u);
         tc_fence_after();
@@ -452,19 +453,21 @@ __device__ void role_mma_chain(const Ctx& cx, const TcParams& prm)
         // Delta^T is complete: its epilogue starts now
         if (elect_one()) mma_commit(cx.bar(B_MMA1_DONE));
         __syncwarp();
-        cx.wait(B_D_READY, j & 1u);
-        // the two output accumulators were read by the output epilogue of chunk j-1, a whole Delta epilogue ago
+        // S0 Q^T runs under the Delta epilogue.  It needs the output accumulators, which the output epilogue of
+        // chunk j-1 has normally released by now, and it has to precede the state update: the state epilogue
+        // overwrites the bf16 state as soon as that update is complete, and completion is in issue order.
         if (j >= 1) cx.wait(B_ACC23_FREE, (j - 1) & 1u);
         tc_fence_after();
-        if (elect_one()) {
-            // S0 Q^T before the state update: the state epilogue overwrites the bf16 state as soon as that update
-            // is complete, and completion is in issue order
-            if (!first) {
+        if (!first && elect_one()) {
 #pragma unroll
-                for (int ks = 0; ks < 8; ++ks)
-                    mma_ts(cx.tmem + TM_ACC2, cx.tmem + TM_SBF + ks * 8,
-                           desc_add(d_q, (ks >> 2) * 16384 + (ks & 3) * 32), ID_SQ, ks > 0);
-            }
+            for (int ks = 0; ks < 8; ++ks)
+                mma_ts(cx.tmem + TM_ACC2, cx.tmem + TM_SBF + ks * 8,
+                       desc_add(d_q, (ks >> 2) * 16384 + (ks & 3) * 32), ID_SQ, ks > 0);
+        }
+        __syncwarp();
+        cx.wait(B_D_READY, j & 1u);
+        tc_fence_after();
+        if (elect_one()) {
 #pragma unroll
             for (int ks = 0; ks < 4; ++ks)
                 mma_ts(cx.tmem + TM_S32, cx.tmem + TM_DPBF + ks * 16, desc_add(d_kn, ks * 2048), ID_DK,
