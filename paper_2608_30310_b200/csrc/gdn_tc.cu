@@ -1042,6 +1042,11 @@ __device__ void role_out(const Ctx& cx, const TcParams& prm, int warp, int lane)
             tmem_ld16(tl + TM_ACC3 + c0, a3);
             if (!first) tmem_ld16(tl + TM_ACC2 + c0, a2);
             tmem_ld_wait();
+            if (g == 3) {
+                // both accumulators have been read: the chain may overwrite them while the last block is stored
+                tc_fence_before();
+                warp_arrive(cx.bar(B_ACC23_FREE), lane);
+            }
             if (og) {
 #pragma unroll
                 for (int i4 = 0; i4 < 4; ++i4) {
@@ -1057,8 +1062,6 @@ __device__ void role_out(const Ctx& cx, const TcParams& prm, int warp, int lane)
                 }
             }
         }
-        tc_fence_before();
-        warp_arrive(cx.bar(B_ACC23_FREE), lane);
         warp_arrive(cx.bar(B_DECAY_FREE0 + (j & 3u)), lane);    // last read of this chunk's decay factors
     }
 }
