@@ -53,7 +53,6 @@ constexpr int LDA = 72;                       // bf16 row stride of the A and X 
 constexpr int LDM = 40;                       // bf16 row stride of the merge scratch (80 B)
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr int kThreads = 896;      // 28 warps, see the role table above (at most 72 registers per thread)
-constexpr int kWgThreads = 256;
 
 // ---- shared memory map (bytes from a 1024-aligned base) ---------------------------------------
 constexpr uint32_t SM_KQ = 0;                 // 3 slots x {2 halves x [128 rows: K 0-63, Q 64-127] x 128 B}  96 KB
@@ -196,7 +195,6 @@ struct ChunkCursor {
     __device__ int row0() const { return row_begin + c * 64; }
     __device__ int nvalid() const { return min(64, row_end - row0()); }
     __device__ bool first() const { return c == 0; }
-    __device__ bool last() const { return c == nchunks - 1; }
 };
 
 struct Ctx {
@@ -248,7 +246,6 @@ struct Ctx {
     }
 };
 
-__device__ __forceinline__ void wg_sync(int id) { asm volatile("bar.sync %0, 256;" ::"r"(id) : "memory"); }
 // One arrival per warp: every lane has fenced its own TMEM / shared-memory accesses, the warp converges,
 // lane 0 arrives.  (A full-warp arrive is 32 serialized shared-memory atomics on one address.)
 __device__ __forceinline__ void warp_arrive(uint32_t bar, int lane)
@@ -295,16 +292,6 @@ __device__ __forceinline__ void tile16_mma_at(float (&c)[2][4], uint32_t a_addr,
     uint32_t a[4], b[4];
     ldm_x4(a, a_addr);
     ldm_x4_trans(b, b_addr);
-    mma_bf16(c[0], a, b[0], b[1]);
-    mma_bf16(c[1], a, b[2], b[3]);
-}
-// c (16 x 16, two 8-column halves) += A[ar0.., ak0..+16) * B[bk0..+16, bn0..+16)
-__device__ __forceinline__ void tile16_mma(float (&c)[2][4], uint32_t a_base, int lda, int ar0, int ak0,
-                                           uint32_t b_base, int ldb, int bk0, int bn0, int lane)
-{
-    uint32_t a[4], b[4];
-    ldm_x4(a, tile_addr(a_base, lda, ar0, ak0, lane));
-    ldm_x4_trans(b, tile_addr(b_base, ldb, bk0, bn0, lane));
     mma_bf16(c[0], a, b[0], b[1]);
     mma_bf16(c[1], a, b[2], b[3]);
 }
@@ -872,7 +859,6 @@ __device__ void role_chain(const Ctx& cx, const TcParams& prm, int wtid)
     const int dv = w4 * 32 + lane;                        // value-dimension index = TMEM lane
     const uint32_t tl = cx.tmem + ((uint32_t)(w4 * 32) << 16);
     Misc* misc = cx.misc;
-    __nv_bfloat16* __restrict__ og = reinterpret_cast<__nv_bfloat16*>(p.out_o);
     const uint32_t num_items = (uint32_t)p.num_seqs * (uint32_t)p.Hv;
     const uint32_t J = count_chunks(prm);
     GDN_TIMERS(long long tt_[16] = {0}; long long tl_ = clock64(); int nch = 0;)
@@ -896,7 +882,7 @@ __device__ void role_chain(const Ctx& cx, const TcParams& prm, int wtid)
         for (int c = 0; c < nchunks; ++c, ++j) {
             const int row0 = row_begin + c * 64;
             const int nvalid = min(64, row_end - row0);
-            const bool first = c == 0, last = c == nchunks - 1;
+            const bool last = c == nchunks - 1;
             const Decay& dc = misc->decay[j & 3u];
             GDN_DBG(const bool dbg = prm.debug && blockIdx.x == 0 && r == 0 && c < 2; float* dbase = prm.debug + c * DBG_STRIDE;)
 
