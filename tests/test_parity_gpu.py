@@ -189,3 +189,26 @@ def test_weak_decay_tail_vs_full_bound_has_teeth(kernel):
         diff = np.linalg.norm(st[0, h] - st_tail[0, h])
         assert diff <= bound + 2 * TOL["bf16"]["state_rel_fro"] * np.linalg.norm(st[0, h])
         assert bound > 0.1                                   # the bound is not vacuous here
+
+
+@pytest.mark.parametrize("kernel", [TC])
+def test_randomised_ragged_batches(kernel):
+    """Seeded sweep over ragged batches: request counts 1-11, lengths 0-330 (plus runs of lengths around one chunk and
+    one long request), seven head configurations, four decay ranges from very weak to very strong.  The pipeline of
+    the tensor-core kernel runs across chain boundaries, so short and empty chains in odd mixes are its edge cases."""
+    rng = np.random.default_rng(2608030310)
+    heads = [(1, 1), (1, 2), (2, 2), (2, 4), (4, 1), (3, 2), (16, 2)]
+    decay = [(-0.1, -0.001), (-2.0, -0.1), (-0.002, -0.0001), (-8.0, -0.4)]
+    for it in range(24):
+        nreq = int(rng.integers(1, 12))
+        lens = [int(x) for x in rng.integers(0, 330, size=nreq)]
+        if it % 7 == 0:
+            lens = [int(x) for x in rng.integers(60, 70, size=nreq)]
+        if it % 11 == 0:
+            lens[0] = int(rng.integers(700, 1500))
+        if sum(lens) == 0:
+            lens[0] = 5
+        hq, g = heads[it % 7]
+        g_lo, g_hi = decay[it % 4]
+        inp = make_inputs(lens, hq, hq * g, 128, 128, "bf16", seed=2608030310 + 50_000 + it, g_lo=g_lo, g_hi=g_hi)
+        check(inp, kernel)
