@@ -126,11 +126,17 @@ int32_t forward(const gdn_desc* d, const void* q, const void* k, const void* v, 
         p.init_state = d->init_state; p.out_o = out_o; p.out_state = out_state;
     }
 
-    if (gdn::launch_scheduler(p.cu, p.num_seqs, sched, stream) != cudaSuccess) return GDN_ERR_CUDA;
-    g_last_launches += 1;
+    const bool use_tc = tc_shape && d->kernel != GDN_KERNEL_FP32_SIMT;
+    // A single request needs no ordering: the tensor-core path then runs without the scheduler kernel, which
+    // matters for the batch-1 state rebuild (one call per layer, a few microseconds each).
+    if (use_tc && p.num_seqs == 1 && gdn::tcgen05_supported(p)) {
+        sched.order = nullptr;
+    } else {
+        if (gdn::launch_scheduler(p.cu, p.num_seqs, sched, stream) != cudaSuccess) return GDN_ERR_CUDA;
+        g_last_launches += 1;
+    }
 
     cudaError_t e = cudaErrorNotSupported;
-    const bool use_tc = tc_shape && d->kernel != GDN_KERNEL_FP32_SIMT;
     if (use_tc) {
         e = gdn::launch_tcgen05(p, sched, stream, &g_last_launches);
         if (e == cudaErrorNotSupported && d->kernel == GDN_KERNEL_TCGEN05) return GDN_ERR_UNSUPPORTED;

@@ -34,12 +34,14 @@ static_assert(sizeof(SchedHeader) == 256, "header is one 256-byte line");
 // concurrent cache hits differ up to 8x in length, so long chains must start first).
 struct Sched {
     SchedHeader* header;
-    int32_t* order;           // [N] request indices, longest first
+    int32_t* order;           // [N] request indices, longest first; null: the requests in the order given (the
+                              // tensor-core path with a single request, which then needs no scheduler kernel)
 };
 
 cudaError_t launch_scheduler(const int32_t* cu, int32_t num_seqs, const Sched& s, cudaStream_t stream);
 cudaError_t launch_simt(const Problem& p, const Sched& s, int io_dtype, cudaStream_t stream, int* launches);
-// Returns cudaErrorNotSupported when the tensor-core path cannot run this problem.
+// Whether the tensor-core path can run this problem; launch_tcgen05 returns cudaErrorNotSupported when it cannot.
+bool tcgen05_supported(const Problem& p);
 cudaError_t launch_tcgen05(const Problem& p, const Sched& s, cudaStream_t stream, int* launches);
 
 }  // namespace gdn

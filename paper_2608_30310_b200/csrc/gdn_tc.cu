@@ -169,7 +169,7 @@ struct ChunkCursor {
     // w = request index.
     __device__ __noinline__ static int4 lookup(const Problem* p, const int32_t* order, uint32_t item)
     {
-        const int n = order[item / p->Hv];
+        const int n = order ? order[item / p->Hv] : (int)(item / p->Hv);       // no order list: requests as given
         const int h = item % p->Hv;
         const int hq = h / (p->Hv / p->Hq);
         return make_int4(p->cu[n], p->cu[n + 1], h | (hq << 16), n);
@@ -1181,9 +1181,14 @@ extern "C" GDN_API void gdn_test_hooks(uint64_t wait_timeout_ns, int32_t skip_kq
     g_skip_kq_load = skip_kq_load_of_chunk;
 }
 
+bool tcgen05_supported(const Problem& p)
+{
+    return p.dk == 128 && p.dv == 128 && p.init_state == nullptr && p.total_tokens > 0;
+}
+
 cudaError_t launch_tcgen05(const Problem& p, const Sched& s, cudaStream_t stream, int* launches)
 {
-    if (p.dk != 128 || p.dv != 128 || p.init_state != nullptr || p.total_tokens <= 0) return cudaErrorNotSupported;
+    if (!tcgen05_supported(p)) return cudaErrorNotSupported;
     CUtensorMap tq, tk, tv;
     if (!make_map(&tq, p.q, (uint64_t)p.total_tokens, (uint64_t)p.Hq * 128) ||
         !make_map(&tk, p.k, (uint64_t)p.total_tokens, (uint64_t)p.Hq * 128) ||

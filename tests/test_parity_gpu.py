@@ -17,7 +17,7 @@ SIMT, TC = 1, 2
 def check(inp, kernel, **kw):
     o, st, launches = run_library(inp, kernel=kernel, **kw)
     ro, rst = oracle.gdn_forward_inputs(inp)
-    assert launches >= 2
+    assert launches >= 1
     return assert_parity(inp, o, st, ro, rst)
 
 
