@@ -89,7 +89,8 @@ enum Bar {
 //   bRest beta e^(G_C - G) / c   (Delta' = Delta~ diag(bRest) accumulates onto the stored state)
 //   rescale / wb: this chunk starts from a rescaled state: the previous chunk's state epilogue multiplies the
 //   stored state by wb = c_prev e^(G_C) first;  cfin = c after this chunk (final state = cfin * stored state)
-struct Decay { float G2[64], beta[64], eG[64], bRest[64], colf[32], colfb[32]; float wb; float G2mid; float cfin; int rescale; };
+struct __align__(16) Decay { float G2[64], beta[64], eG[64], bRest[64], colf[32], colfb[32]; float wb; float G2mid; float cfin; int rescale; int nvalid; };
+static_assert(sizeof(Decay) % 16 == 0, "the decay ring is read with 16-byte vector loads");
 struct Misc {
     float ones[64];
     Decay decay[4];                    // per-chunk decay factors, ring of 4 (decay warp writes; pre and chain read)
@@ -490,7 +491,8 @@ __device__ void role_decay(const Ctx& cx, const TcParams& prm)
         const float g1 = ok1 ? p.g[(size_t)(row0 + lane + 32) * p.Hv + h] : 0.f;
         const float b0 = ok0 ? p.beta[(size_t)(row0 + lane) * p.Hv + h] : 0.f;
         const float b1 = ok1 ? p.beta[(size_t)(row0 + lane + 32) * p.Hv + h] : 0.f;
-        float G0 = g0 * kLog2e, G1 = g1 * kLog2e;
+        // clamped so that g = -inf (alpha = 0) keeps every difference of cumulative sums finite; 2^-1e5 is still 0
+        float G0 = fmaxf(g0 * kLog2e, -1.0e5f), G1 = fmaxf(g1 * kLog2e, -1.0e5f);
 #pragma unroll
         for (int off = 1; off < 32; off <<= 1) {
             const float u0 = __shfl_up_sync(0xffffffffu, G0, off), u1 = __shfl_up_sync(0xffffffffu, G1, off);
@@ -514,7 +516,7 @@ __device__ void role_decay(const Ctx& cx, const TcParams& prm)
         const float G31 = __shfl_sync(0xffffffffu, G0, 31);
         const float cf = ex2_approx(G31 - G0);
         dc.colf[lane] = cf; dc.colfb[lane] = cf * b0;
-        if (lane == 0) { dc.wb = cprev * eGC; dc.G2mid = G31; dc.cfin = c; dc.rescale = rescale ? 1 : 0; }
+        if (lane == 0) { dc.wb = cprev * eGC; dc.G2mid = G31; dc.cfin = c; dc.rescale = rescale ? 1 : 0; dc.nvalid = nvalid; }
         warp_arrive(cx.bar(B_DECAY_READY0 + (j & 3u)), lane);
     }
 }
@@ -555,7 +557,9 @@ __device__ void role_g1(const Ctx& cx, const TcParams& prm, int wtid)
         // Delta epilogue, so that P^ itself is one MMA operand and its column-scaled copy the other
         const float* __restrict__ colscale = isA ? dc.beta : misc->ones;
         const float* __restrict__ colfac = isA ? dc.colfb : dc.colf;
-        const int t_lim = isA ? t : t + 1;                      // keep columns s < t_lim
+        // keep columns s < t_lim; rows past the end of the request (whose k, q may be anything) are zeroed
+        const bool row_ok = t < dc.nvalid;
+        const int t_lim = row_ok ? (isA ? t : t + 1) : 0;
         cx.wait(B_GRAM_DONE, c & 1u);
         tc_fence_after();
         // buffers: P of chunk c was last read by the MMAs of chunk c-3, A by the solve of chunk c-2
@@ -566,7 +570,7 @@ __device__ void role_g1(const Ctx& cx, const TcParams& prm, int wtid)
         // column blocks are dealt so that each warp of a lane window gets one block that touches the
         // diagonal and one that does not: half 0 -> blocks {0, 2}, half 1 -> blocks {1, 3}
         const bool lower_rows = (w4 & 1) != 0;                  // rows 32-63
-        const float rowf = lower_rows ? ex2_approx(G2t - dc.G2mid) : 0.f;
+        const float rowf = (lower_rows && row_ok) ? ex2_approx(G2t - dc.G2mid) : 0.f;
 #pragma unroll 1
         for (int g = 0; g < 2; ++g) {
             const int cb = hf + 2 * g, c0 = 16 * cb;
@@ -921,6 +925,7 @@ __device__ void role_chain(const Ctx& cx, const TcParams& prm, int wtid)
             }
             tmem_st_wait();
             tc_fence_before();
+            const float cfin = dc.cfin;          // read before the arrival below lets the pipeline move on to the slot's reuse
             warp_arrive(cx.bar(B_D_READY), lane);
             GDN_T(2);
 
@@ -933,7 +938,6 @@ __device__ void role_chain(const Ctx& cx, const TcParams& prm, int wtid)
                 wb = misc->decay[(j + 1) & 3u].wb;
                 rescale = misc->decay[(j + 1) & 3u].rescale != 0;
             }
-            const float cfin = dc.cfin;
             cx.wait(B_STATE_DONE, j & 1u);
             GDN_T(3);
             tc_fence_after();

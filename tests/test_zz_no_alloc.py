@@ -14,8 +14,9 @@ import ctypes
 import numpy as np
 import pytest
 
+import oracle
 from gdn_workloads import make_inputs
-from gpu_utils import run_library, TOL, state_rel_fro
+from gpu_utils import run_library, assert_parity, TOL, state_rel_fro
 
 pytestmark = pytest.mark.gpu
 
@@ -35,6 +36,26 @@ def test_static_scratch_matches_workspace_entry_twice(io, dk, kernel):
         assert state_rel_fro(st_new, st_ref)[0] <= tol["state_rel_fro"]
         np.testing.assert_array_equal(o_new, o_ref)        # same kernels, same order: bitwise equal
         np.testing.assert_array_equal(st_new, st_ref)
+        ro, rst = oracle.gdn_forward_inputs(inp)             # and directly against the oracle
+        assert_parity(inp, o_new, st_new, ro, rst)
+
+
+def test_static_scratch_at_its_request_limit_and_with_one_request():
+    """4,096 requests fill the built-in array to its last byte (the order list ends exactly there); a single
+    request on the tensor-core path runs without the scheduler kernel, i.e. without touching the array."""
+    lens = [(i * 7) % 4 for i in range(4096)]              # lengths 0..3
+    inp = make_inputs(lens, 1, 2, 64, 64, "f32", seed=303)
+    o_ref, st_ref, _ = run_library(inp, fn="gdn_tail_replay")
+    o_new, st_new, _ = run_library(inp, fn="gdn_tail_replay_static_scratch")
+    np.testing.assert_array_equal(o_new, o_ref)
+    np.testing.assert_array_equal(st_new, st_ref)
+    ro, rst = oracle.gdn_forward_inputs(inp)
+    assert_parity(inp, o_new, st_new, ro, rst)
+    one = make_inputs([200], 2, 4, 128, 128, "bf16", seed=304)
+    o1, st1, launches = run_library(one, fn="gdn_tail_replay_static_scratch")
+    assert launches == 1
+    ro, rst = oracle.gdn_forward_inputs(one)
+    assert_parity(one, o1, st1, ro, rst)
 
 
 def test_static_scratch_rejects_oversize_and_host_memory():
