@@ -13,6 +13,7 @@ from gpu_utils import run_library, assert_parity, assert_parity_lean, state_rel_
 pytestmark = pytest.mark.gpu
 
 SIMT, TC = 1, 2
+TC_SINGLE, TC_PAIR = 3, 4          # the tensor-core path with its work split fixed: one chain / a sibling pair per CTA
 
 
 def check(inp, kernel, **kw):
@@ -54,26 +55,60 @@ def test_simt_init_state_resume():
     assert np.abs(o_tail - ro[120:]).max() < 1e-4
 
 
-@pytest.mark.parametrize("kernel", [SIMT, TC, 0])
+@pytest.mark.parametrize("kernel", [SIMT, TC, TC_SINGLE, TC_PAIR, 0])
 def test_bf16_d128_ragged_batch(kernel):
     lens = [130, 64, 1, 0, 63, 65, 127, 128, 129, 410, 5]
     inp = make_inputs(lens, 2, 4, 128, 128, "bf16", seed=77)
     check(inp, kernel)
 
 
-@pytest.mark.parametrize("kernel", [SIMT, TC])
+@pytest.mark.parametrize("kernel", [SIMT, TC, TC_PAIR])
 def test_config1_single_layer(kernel):
     check(config_single_layer(), kernel)
 
 
-@pytest.mark.parametrize("kernel", [TC])
+@pytest.mark.parametrize("kernel", [TC, TC_SINGLE, TC_PAIR])
 def test_gqa_group_sizes(kernel):
-    for Hq, Hv in [(1, 1), (1, 4), (3, 3), (2, 6)]:
+    for Hq, Hv in [(1, 1), (1, 4), (3, 3), (2, 6), (2, 8)]:
+        if kernel == TC_PAIR and (Hv // Hq) % 2:
+            continue                                       # pairs need an even number of v-heads per q/k head
         inp = make_inputs([200, 77], Hq, Hv, 128, 128, "bf16", seed=5 + Hq * 10 + Hv)
         check(inp, kernel)
 
 
-@pytest.mark.parametrize("kernel", [SIMT, TC])
+@pytest.mark.parametrize("kernel", [TC_SINGLE, TC_PAIR])
+def test_tc_init_state_resume_ragged(kernel):
+    """Resume identity on the tensor-core path: run(prefix + tail) == run(tail, init = run(prefix)), request by
+    request on a ragged batch that includes empty tails (whose final state must equal the start state) and
+    tails shorter than a chunk; the resumed outputs and states are also compared with the oracle."""
+    lens = [200, 64, 0, 1, 129, 330, 63, 0]
+    cut = [120, 64, 0, 0, 1, 200, 10, 0]                   # rows of each request that form the prefix
+    inp = make_inputs(lens, 2, 4, 128, 128, "bf16", seed=23)
+    pre_lens = cut
+    tail_lens = [l - c for l, c in zip(lens, cut)]
+    def split(lens_part, offs):
+        rows = np.concatenate([np.arange(int(inp.cu_tail_lens[n]) + o, int(inp.cu_tail_lens[n]) + o + l)
+                               for n, (l, o) in enumerate(zip(lens_part, offs))]).astype(np.int64)
+        sub = make_inputs(lens_part, 2, 4, 128, 128, "bf16", seed=1)
+        for name in ("q", "k", "v", "g", "beta", "q_bits", "k_bits", "v_bits"):
+            setattr(sub, name, np.ascontiguousarray(getattr(inp, name)[rows]))
+        return sub, rows
+    pre, _ = split(pre_lens, [0] * len(lens))
+    tail, tail_rows = split(tail_lens, cut)
+    ro, rst = oracle.gdn_forward_inputs(inp)
+    _, st_pre, _ = run_library(pre, kernel=kernel)
+    o_tail, st_res, _ = run_library(tail, kernel=kernel, init_state=st_pre, canary=True)
+    assert_parity(inp, None, st_res, None, rst)
+    assert np.abs(o_tail - ro[tail_rows]).max() <= TOL["bf16"]["o_max_abs"]
+    # and against the oracle started from the same (GPU-made, fp32) prefix state
+    ro2, rst2 = oracle.gdn_forward_inputs(tail, init_state=st_pre.astype(np.float32).astype(np.float64))
+    assert_parity(tail, o_tail, st_res, ro2, rst2)
+    for n, l in enumerate(tail_lens):
+        if l == 0:
+            np.testing.assert_array_equal(st_res[n], st_pre[n].astype(np.float32).astype(np.float64))
+
+
+@pytest.mark.parametrize("kernel", [SIMT, TC_SINGLE, TC_PAIR])
 def test_run_to_run_bitwise_determinism(kernel):
     inp = make_inputs([100, 37, 200], 2, 4, 128, 128, "bf16", seed=9)
     o1, s1, _ = run_library(inp, kernel=kernel)
@@ -82,7 +117,7 @@ def test_run_to_run_bitwise_determinism(kernel):
     np.testing.assert_array_equal(s1, s2)
 
 
-@pytest.mark.parametrize("kernel", [SIMT, TC])
+@pytest.mark.parametrize("kernel", [SIMT, TC_SINGLE, TC_PAIR])
 def test_guard_rows_around_outputs_stay_untouched(kernel):
     """out_o sits between 64 guard rows on each side and out_state between two guard states, all filled with a
     bit pattern; ragged last chunks (whose 64-row tiles reach past the request and past the end of the batch)
@@ -116,7 +151,7 @@ def _poison_other_requests(inp, keep):
     return p
 
 
-@pytest.mark.parametrize("kernel", [SIMT, TC])
+@pytest.mark.parametrize("kernel", [SIMT, TC_SINGLE, TC_PAIR])
 def test_poisoned_neighbour_rows_do_not_leak(kernel):
     """The 64-row tiles of a request's ragged last chunk overlap the first rows of the next request (and a
     short request sits inside tiles of its neighbours).  Filling every foreign row with large finite values
@@ -150,7 +185,7 @@ def test_host_memory_call(kernel):
     assert_parity(inp, o, st, ro, rst)
 
 
-@pytest.mark.parametrize("kernel", [SIMT, TC])
+@pytest.mark.parametrize("kernel", [SIMT, TC_SINGLE, TC_PAIR])
 def test_strong_decay_and_beta_zero(kernel):
     """alpha -> 0 keeps only the last token's rank-1 update; beta = 0 keeps the state at zero."""
     inp = make_inputs([130], 1, 2, 128, 128, "bf16", seed=41)
@@ -162,15 +197,22 @@ def test_strong_decay_and_beta_zero(kernel):
     inp.beta[:] = 0.0
     o, st, _ = run_library(inp, kernel=kernel)
     assert np.all(st == 0) and np.all(o == 0)
+    # alpha = 0 exactly (g = -inf) on single tokens: inside a chunk, on a chunk's first and on its last token
+    inp = make_inputs([200], 1, 2, 128, 128, "bf16", seed=44)
+    for t, h in ((37, 0), (64, 1), (127, 0), (128, 1)):
+        inp.g[t, h] = -np.inf
+    o, st, _ = run_library(inp, kernel=kernel)
+    ro, rst = oracle.gdn_forward_inputs(inp)
+    assert_parity(inp, o, st, ro, rst)
 
 
-@pytest.mark.parametrize("kernel", [SIMT, TC])
+@pytest.mark.parametrize("kernel", [SIMT, TC_SINGLE, TC_PAIR])
 def test_weak_decay_long_memory(kernel):
     inp = make_inputs([700], 1, 2, 128, 128, "bf16", seed=43, g_lo=-0.002, g_hi=-0.0001)
     check(inp, kernel)
 
 
-@pytest.mark.parametrize("kernel", [TC])
+@pytest.mark.parametrize("kernel", [TC, TC_SINGLE])
 def test_config3_concurrent_hits_full_size_all_chains(kernel):
     """Full-size 32-request batch in the benchmark's launch configuration: every one of the 1,024 chains
     (all outputs, all final states) against the oracle."""
@@ -249,7 +291,7 @@ def test_weak_decay_tail_vs_full_bound_has_teeth(kernel):
         assert bound > 0.1                                   # the bound is not vacuous here
 
 
-@pytest.mark.parametrize("kernel", [TC])
+@pytest.mark.parametrize("kernel", [TC_SINGLE, TC_PAIR])
 def test_randomised_ragged_batches(kernel):
     """Seeded sweep over ragged batches: request counts 1-11, lengths 0-330 (plus runs of lengths around one chunk and
     one long request), seven head configurations, four decay ranges from very weak to very strong.  The pipeline of
@@ -267,6 +309,8 @@ def test_randomised_ragged_batches(kernel):
         if sum(lens) == 0:
             lens[0] = 5
         hq, g = heads[it % 7]
+        if kernel == TC_PAIR and g % 2:
+            g += 1                                         # pairs need an even number of v-heads per q/k head
         g_lo, g_hi = decay[it % 4]
         inp = make_inputs(lens, hq, hq * g, 128, 128, "bf16", seed=2608030310 + 50_000 + it, g_lo=g_lo, g_hi=g_hi)
         check(inp, kernel)
