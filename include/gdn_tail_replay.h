@@ -75,11 +75,7 @@ typedef enum { GDN_MEM_DEVICE = 0, GDN_MEM_HOST = 1 } gdn_memory;
 typedef enum {
     GDN_KERNEL_AUTO = 0,        /* tensor-core path when the shape allows it, else the fp32 path */
     GDN_KERNEL_FP32_SIMT = 1,   /* token-recurrent, all-fp32 FFMA; any supported shape and dtype */
-    GDN_KERNEL_TCGEN05 = 2,     /* chunkwise WY form on tcgen05/TMEM; bf16, dk = dv = 128, chunk 64 */
-    /* The tensor-core path with its work split fixed instead of chosen from the chain count: */
-    GDN_KERNEL_TCGEN05_SINGLE = 3,  /* one chain (request, v-head) per CTA at a time */
-    GDN_KERNEL_TCGEN05_PAIR = 4     /* the two v-heads that share a q/k head per CTA, interleaved chunk by chunk
-                                       (needs an even number of v-heads per q/k head, else UNSUPPORTED) */
+    GDN_KERNEL_TCGEN05 = 2      /* chunkwise WY form on tcgen05/TMEM; bf16, dk = dv = 128, chunk 64 */
 } gdn_kernel;
 
 typedef struct gdn_desc {

@@ -13,7 +13,6 @@ GDN_OK = 0
 GDN_F32, GDN_BF16 = 0, 1
 GDN_MEM_DEVICE, GDN_MEM_HOST = 0, 1
 GDN_KERNEL_AUTO, GDN_KERNEL_FP32_SIMT, GDN_KERNEL_TCGEN05 = 0, 1, 2
-GDN_KERNEL_TCGEN05_SINGLE, GDN_KERNEL_TCGEN05_PAIR = 3, 4
 
 
 class GdnError(RuntimeError):

@@ -71,12 +71,10 @@ int32_t forward(const gdn_desc* d, const void* q, const void* k, const void* v, 
                          (d->head_v_dim == 64 || d->head_v_dim == 128);
     if (!dims_ok) return GDN_ERR_UNSUPPORTED;
     if (chunk != 64) return GDN_ERR_UNSUPPORTED;
-    const bool tc_kernel = d->kernel == GDN_KERNEL_TCGEN05 || d->kernel == GDN_KERNEL_TCGEN05_SINGLE ||
-                           d->kernel == GDN_KERNEL_TCGEN05_PAIR;
-    if (d->kernel != GDN_KERNEL_AUTO && d->kernel != GDN_KERNEL_FP32_SIMT && !tc_kernel) return GDN_ERR_INVALID_ARG;
+    if (d->kernel != GDN_KERNEL_AUTO && d->kernel != GDN_KERNEL_FP32_SIMT && d->kernel != GDN_KERNEL_TCGEN05)
+        return GDN_ERR_INVALID_ARG;
     const bool tc_shape = d->io_dtype == GDN_BF16 && d->head_k_dim == 128 && d->head_v_dim == 128;
-    if (tc_kernel && !tc_shape) return GDN_ERR_UNSUPPORTED;
-    if (d->kernel == GDN_KERNEL_TCGEN05_PAIR && ((d->num_v_heads / d->num_qk_heads) & 1)) return GDN_ERR_UNSUPPORTED;
+    if (d->kernel == GDN_KERNEL_TCGEN05 && !tc_shape) return GDN_ERR_UNSUPPORTED;
     if (d->num_seqs == 0) return GDN_OK;
     const size_t need = gdn_workspace_size(d);
     if (!d->workspace || d->workspace_bytes < need) return GDN_ERR_WORKSPACE;
@@ -139,9 +137,8 @@ int32_t forward(const gdn_desc* d, const void* q, const void* k, const void* v, 
 
     cudaError_t e = cudaErrorNotSupported;
     if (use_tc) {
-        const int pairing = d->kernel == GDN_KERNEL_TCGEN05_SINGLE ? 1 : d->kernel == GDN_KERNEL_TCGEN05_PAIR ? 2 : 0;
-        e = gdn::launch_tcgen05(p, sched, pairing, stream, &g_last_launches);
-        if (e == cudaErrorNotSupported && tc_kernel) return GDN_ERR_UNSUPPORTED;
+        e = gdn::launch_tcgen05(p, sched, stream, &g_last_launches);
+        if (e == cudaErrorNotSupported && d->kernel == GDN_KERNEL_TCGEN05) return GDN_ERR_UNSUPPORTED;
     }
     if (e == cudaErrorNotSupported) e = gdn::launch_simt(p, sched, d->io_dtype, stream, &g_last_launches);
     if (e == cudaErrorNotSupported) return GDN_ERR_UNSUPPORTED;

@@ -42,7 +42,6 @@ cudaError_t launch_scheduler(const int32_t* cu, int32_t num_seqs, const Sched& s
 cudaError_t launch_simt(const Problem& p, const Sched& s, int io_dtype, cudaStream_t stream, int* launches);
 // Whether the tensor-core path can run this problem; launch_tcgen05 returns cudaErrorNotSupported when it cannot.
 bool tcgen05_supported(const Problem& p);
-// pairing: 0 = decide from the chain count, 1 = one chain per CTA, 2 = the two v-heads of a q/k head per CTA
-cudaError_t launch_tcgen05(const Problem& p, const Sched& s, int pairing, cudaStream_t stream, int* launches);
+cudaError_t launch_tcgen05(const Problem& p, const Sched& s, cudaStream_t stream, int* launches);
 
 }  // namespace gdn

@@ -1,45 +1,46 @@
 // Tensor-core path of the GDN forward: chunkwise WY (UT-transform) evaluation of Eq. 1 on
 // tcgen05 MMAs with TMEM accumulators and TMA-staged bf16 tiles.  bf16 io, dk = dv = 128, chunk 64.
 //
-// Everything is kept in the transposed orientation so that every tcgen05 MMA has M = 128 (one TMEM lane
-// per value-dimension index i): the carried state is S (dv x dk, fp32, TMEM-resident), and per chunk of
-// C = 64 tokens with start state S0:
+// Everything is kept in the transposed orientation so that every MMA has M = 128 (one TMEM lane
+// per value-dimension index i, or per key-dimension index for W^T): the carried state is
+// S (dv x dk, fp32, TMEM-resident), and per chunk of C = 64 tokens with start state S0:
 //
 //   G_t   = cumsum(g) inside the chunk;  Gam[t,s] = exp(G_t - G_s) (t >= s)
-//   Gram  = [K;Q] K^T                        (tcgen05, 128 x 64: rows 0-63 K K^T, rows 64-127 Q K^T)
-//   A^    = strict_lower(Gam (K K^T)) diag(beta),  P = lower_incl(Gam (Q K^T))
-//   P^    = (I + A^)^-1                       (8 x 8 diagonal blocks by substitution in fp32, block merges on
-//                                              mma.sync bf16; built in place, in MMA operand layout)
-//           With beta on the columns, (I + A)^-1 diag(beta) = diag(beta) P^ for A = diag(beta) strict_lower(..):
-//           P^ itself is an MMA operand and the row factor beta is applied in the Delta epilogue.
-//   W~^T  = K^T (P^ diag(e^G))^T              (mma.sync, 128(dk) x 64, e^G folded into the K fragments)
-//   Dl^T  = (V^T P^^T - S0 W~^T) diag(beta)   (two tcgen05 MMAs into one accumulator, second negated)
-//   O^T   = (S0 Q^T) diag(e^G) + Dl^T P^T     (S0 Q^T is scaled in place in its accumulator, then the second
-//                                              product accumulates on top)
-//   S     = e^{G_C} S0 + (Dl diag(e^{G_C - G}))^T K    (tcgen05, accumulating in place: tensor memory holds S / c
-//                                              with c the running product of the chunk decays, folded into the
+//   Gram  = [K;Q] K^T                        (MMA, 128 x 64: rows 0-63 K K^T, rows 64-127 Q K^T)
+//   A     = strict_lower(beta_t Gam (K K^T)) and X = (I + A)^-1 enter as T' = X diag(beta), T'' = X diag(beta e^G).
+//           With beta moved to the columns, A^ = strict_lower(Gam (K K^T)) diag(beta) and P^ = (I + A^)^-1 (8 x 8
+//           diagonal blocks by substitution in fp32, block merges on mma.sync bf16 with ldmatrix-fed fragments), one
+//           has T' = diag(beta) P^ and T'' = diag(beta) P^ diag(e^G): P^ itself and its column-scaled copy
+//           P^ diag(e^G) are the two MMA operands, and the common row factor beta moves behind the products
+//   P     = lower_incl(Gam (Q K^T)) diag(beta)    (beta on the columns here as well)
+//   W~^T  = K^T (P^ diag(e^G))^T              (MMA, 128(dk) x 64)
+//   Dl~^T = V^T P^^T - S0 W~^T                (two MMAs into one accumulator, second negated; Delta = Dl~ diag(beta))
+//   O^T   = (S0 Q^T) diag(e^G) + Dl~^T P^T    (two MMAs, combined in the epilogue)
+//   S     = e^{G_C} S0 + (Dl~ diag(beta e^{G_C - G}))^T K   (MMA accumulating in place: tensor memory holds S / c with
+//                                              c the running product of the chunk decays, folded into the
 //                                              per-token factors; rescaled before c drops below 2^-40)
 //
-// A CTA works on one item at a time: one chain (request, v-head), or the two chains of a request whose
-// v-heads share a q/k head ("pair").  A pair shares every K/Q tile and the raw Gram product, keeps both
-// fp32 states in tensor memory and alternates between its chains chunk by chunk: consecutive steps of the
-// CTA then belong to independent recurrences, so one chain's epilogues overlap the other chain's MMAs and
-// the bf16 copy of a state is made while the other chain computes.  A step = one chunk of one chain.
-//
-// The CTA is warp-specialised and software-pipelined over its steps (28 warps):
-//   warp 0       TMA producer: K/Q tiles (3 slots, one per chunk of an item), V tiles (2 slots, one per step)
-//   warp 1       issues the chain MMAs of each step (U^T, S0 W~^T, S0 Q^T, state update, Dl^T P^T)
-//   warp 2       issues the Gram MMA of each K/Q tile
-//   warp 3       decay warp: loads g and beta ahead, scans the log-decay, publishes the per-step factors
-//   warps 4-15   three pre-stage teams of four warps; team T takes steps T, T+3, ..: Gram post-processing
-//                (A^ and P), the triangular solve in place, W~^T.  One code path shared by twelve warps.
-//   warps 16-23  chain group: Delta epilogue, bf16 copy of the next step's start state (rescaling when due),
-//                start states from init_state, final states
-//   warps 24-27  output group: scales S0 Q^T in place, then reads O^T and stores the valid rows
-// Items are ordered longest-first by the scheduler kernel and dealt to CTAs in snake order, so each role
-// walks its CTA's step sequence without any broadcast.  Padding rows of a ragged last chunk get g = 0,
-// beta = 0 and zero rows in A^ and P, which makes them inert; their outputs are not stored.
-// Every mbarrier wait is bounded: on expiry the CTA records GDN_ERR_TIMEOUT, stops storing and unwinds.
+// The CTA is warp-specialised and software-pipelined over the chunks of all chains it owns (28 warps):
+//   warp 0       TMA producer: K/Q tiles three chunks ahead (4 slots), V one chunk ahead (1 slot)
+//   warp 1       issues the chain MMAs (U^T, S0 W^T, the state update, then S0 Q^T and Dl~^T P^T)
+//   warp 2       issues the Gram MMAs, ahead of the chain
+//   warp 3       decay warp: loads g and beta up to three chunks ahead, scans the log-decay and publishes the
+//                per-chunk decay factors
+//   warps 4-11   group G1 (two warps per TMEM lane window): Gram post-processing of chunk k+1 (A^ straight into the
+//                chunk's T' buffer, P into its P buffer, both in MMA operand layout), then the W^T epilogue of chunk k
+//   warps 12-19  chain group: Delta epilogue, state conversion (and rescaling when due), start states from
+//                init_state, final states
+//   warps 20-23  group G2, two teams of two warps that take alternate chunks: the triangular solve in place in the T'
+//                buffer, then the column-scaled copy T''; the team then issues the W^T MMA itself
+//   warps 24-27  output group: output epilogue of chunk j, off the chain's critical path
+// Every per-chunk loop is kept rolled with 16-column TMEM accesses: straight-line code larger than the
+// instruction caches runs at a fraction of the issue rate, so the static footprint matters as much as the
+// instruction count.
+// Chains (request, v-head) are ordered longest-first by the scheduler kernel and dealt to CTAs in
+// snake order, so each role can walk its CTA's chunk sequence without any broadcast.  Padding rows
+// of a ragged last chunk get beta = 0 and a cumulative decay that makes their rows of A^ and P vanish, which keeps
+// them inert whatever (finite) values follow the request in memory; their outputs are not stored.
+// Every mbarrier wait is bounded: on expiry the CTA records GDN_ERR_TIMEOUT and unwinds.
 #include <cuda.h>
 #include "common.cuh"
 #include "ptx.cuh"
@@ -49,75 +50,73 @@ namespace {
 
 using namespace ptx;
 
+constexpr int LDM = 40;                       // bf16 row stride of the merge scratch (80 B: conflict-free ldmatrix)
 constexpr float kLog2e = 1.4426950408889634f;
-constexpr int kThreads = 896;                 // 28 warps, see the role table above (at most 72 registers per thread)
-constexpr int kTeams = 3;
-constexpr uint32_t RD = 8;                    // depth of the decay ring (steps)
-constexpr uint32_t RTP = 3, RP = 4;           // depths of the P^ and P operand rings (steps)
-static_assert(RTP == kTeams, "the P^ ring barriers double as per-team barriers");
+constexpr int kThreads = 896;      // 28 warps, see the role table above (at most 72 registers per thread)
 
 // ---- shared memory map (bytes from a 1024-aligned base) ---------------------------------------
-constexpr uint32_t SM_KQ = 0;                 // 3 slots x {2 halves x [128 rows: K 0-63, Q 64-127] x 128 B}  96 KB
+constexpr uint32_t SM_KQ = 0;                 // 4 slots x {2 halves x [128 rows: K 0-63, Q 64-127] x 128 B} 128 KB
 constexpr uint32_t KQ_SLOT = 32768;
-constexpr uint32_t SM_V = 98304;              // 2 slots x {2 halves x [64 rows] x 128 B}                    32 KB
-constexpr uint32_t V_SLOT = 16384;
-constexpr uint32_t SM_WT = 131072;            // W~^T [dk][t] bf16, 128 rows x 128 B                         16 KB
-constexpr uint32_t SM_TP = 147456;            // RTP x P^ [t][s] bf16 (A^ first, inverted in place)          24 KB
-constexpr uint32_t SM_P = SM_TP + RTP * 8192; // RP x P [t][s] bf16                                          32 KB
-constexpr uint32_t SM_MH = SM_P + RP * 8192;  // merge scratch of the solve: 512 B per pre-stage warp         6 KB
-constexpr uint32_t SM_MISC = ((SM_MH + kTeams * 4 * 512 + 1023) / 1024) * 1024;
+constexpr uint32_t NKQ = 4;
+constexpr uint32_t SM_V = SM_KQ + NKQ * KQ_SLOT;   // 2 halves x [64 rows] x 128 B                          16 KB
+constexpr uint32_t SM_WT = SM_V + 16384;      // W^T [dk][t] bf16, 128 rows x 128 B                          16 KB
+constexpr uint32_t SM_TP = SM_WT + 16384;     // 3 x T' [t][s] bf16: A^ from the post-processing, inverted in place  24 KB
+constexpr uint32_t SM_TPP = SM_TP + 3 * 8192; // T'' [t][s] bf16 (one buffer)                                  8 KB
+constexpr uint32_t SM_P = SM_TPP + 8192;      // 3 x P [t][s] bf16                                           24 KB
+constexpr uint32_t SM_MH = SM_P + 3 * 8192;   // merge scratch of the solve, bf16 [32][LDM]
+constexpr uint32_t MH_BYTES = 32 * LDM * 2;   // one per solve team
+constexpr uint32_t SM_MISC = ((SM_MH + 2 * MH_BYTES + 15) / 16) * 16;
 
 enum Bar {
-    B_FULL_KQ0 = 0, B_KQ_FREE0 = 3, B_FULL_V0 = 6, B_V_FREE0 = 8, B_GRAM_DONE0 = 10, B_GRAM_FREE = 13,
-    B_DECAY_READY0, B_DECAY_FREE0 = B_DECAY_READY0 + RD, B_TP_FREE0 = B_DECAY_FREE0 + RD, B_TP_READY0 = B_TP_FREE0 + RTP,
-    B_P_FREE0 = B_TP_READY0 + RTP, B_PRE_DONE0 = B_P_FREE0 + RP, B_WT_FREE0 = B_PRE_DONE0 + 3, B_MMA1_DONE = B_WT_FREE0 + 3,
-    B_SQ_DONE, B_D_READY, B_STATE_DONE, B_SBF_READY, B_ACC2_SCALED, B_ACC2_FREE, B_MMA3_DONE, NUM_BARS
+    B_FULL_KQ0 = 0, B_FULL_KQ1, B_FULL_KQ2, B_FULL_KQ3, B_FULL_V, B_GRAM_DONE, B_W_DONE0, B_W_DONE1, B_U_DONE, B_MMA1_DONE,
+    B_MMA3_DONE, B_STATE_DONE, B_KQ_FREE0, B_KQ_FREE1, B_KQ_FREE2, B_KQ_FREE3, B_P_FREE0, B_P_FREE1, B_P_FREE2,
+    B_TP_FREE0, B_TP_FREE1, B_TP_FREE2,
+    B_GRAM_READ, B_WACC_READ,
+    B_PRE_DONE0, B_PRE_DONE1, B_D_READY, B_SBF_READY, B_ACC23_FREE, B_SQ_DONE,
+    B_DECAY_READY0, B_DECAY_READY1, B_DECAY_READY2, B_DECAY_READY3,
+    B_DECAY_FREE0, B_DECAY_FREE1, B_DECAY_FREE2, B_DECAY_FREE3,
+    B_A_READY0, B_A_READY1, B_A_READY2, B_TP_READY0, B_TP_READY1, B_TP_READY2, NUM_BARS
 };
-// A waiter may only wait for phase k of an mbarrier once it knows phase k - 1 complete (a parity wait cannot tell
-// "two phases behind" from "done"), and arrivals of phase k + 1 must not start before phase k is complete.  Barriers
-// that the three pre-stage teams wait on or arrive at are therefore kept per team (GRAM_DONE, PRE_DONE, WT_FREE,
-// and the P^ ring, whose depth equals the number of teams): every team then sees consecutive phases of its own.
 
-// Per-step decay factors.  The fp32 state lives in tensor memory divided by a running factor c (the product of
+// colf[s] = 2^(G2_31 - G2_s), s < 32: column factors of the purely off-diagonal quadrant of Gam
+// Per-chunk decay factors.  The fp32 state lives in tensor memory divided by a running factor c (the product of
 // the chunk decays since the last rescale), so that a chunk update is a plain accumulation; c is folded into
 // the factors below, and the state is rescaled (c back to 1) before c leaves [2^-40, 1].
 //   G2    log2-domain inclusive cumulative decay,  beta
-//   colf  2^(G2[31] - G2[s]) for s < 32,  colfb = colf * beta[s]   (off-diagonal quadrant of Gam is rank 1)
-//   eG    e^G c_prev         (column factors of W~^T, so that it comes out multiplied by c_prev, as
-//                             S0 = c_prev * stored state; also the factor of (stored state) q in the outputs)
+//   colf  2^(G2[31] - G2[s]) for s < 32,  colfb = colf * beta[s]
+//   eG    e^G c_prev         (column factors of T'', so that W^T comes out multiplied by c_prev, as
+//                             S0 = c_prev * stored state; also the output epilogue's factor of (stored state) q)
 //   bRest beta e^(G_C - G) / c   (Delta' = Delta~ diag(bRest) accumulates onto the stored state)
-//   rescale / wb: this step starts from a rescaled state: whoever prepares the step's start state multiplies
-//   the stored state by wb = c_prev e^(G_C) first;  cfin = c after this step (final state = cfin * stored state)
-struct __align__(16) Decay {
-    float G2[64], beta[64], eG[64], bRest[64], colf[32], colfb[32];
-    float wb, G2mid, cfin; int rescale; int nvalid; int pad[3];
-};
+//   rescale / wb: this chunk starts from a rescaled state: the previous chunk's state epilogue multiplies the
+//   stored state by wb = c_prev e^(G_C) first;  cfin = c after this chunk (final state = cfin * stored state)
+struct __align__(16) Decay { float G2[64], beta[64], eG[64], bRest[64], colfb[32]; float wb; float G2mid; float cfin; int rescale; int pad[3]; };
 static_assert(sizeof(Decay) % 16 == 0, "the decay ring is read with 16-byte vector loads");
 struct Misc {
-    float ones[64];
-    Decay decay[RD];
+    Decay decay[4];                    // per-chunk decay factors, ring of 4 (decay warp writes; pre and chain read)
     unsigned long long bars[NUM_BARS];
     uint32_t tmem_base;
     volatile uint32_t abort;
     unsigned long long timeout_ns;
 };
-constexpr uint32_t SM_TOTAL = SM_MISC + ((sizeof(Misc) + 1023) / 1024) * 1024;
-constexpr uint32_t SMEM_BYTES = SM_TOTAL + 1024;   // slack for the manual 1024-byte alignment
+constexpr uint32_t SM_TOTAL = SM_MISC + ((sizeof(Misc) + 15) / 16) * 16;
+constexpr uint32_t SMEM_BYTES = SM_TOTAL + 1008;   // slack for the manual 1024-byte alignment of a 16-byte aligned base
 static_assert(SMEM_BYTES <= 232448, "exceeds the 227 KB shared memory of one CTA");
 
 // ---- TMEM column map (512 columns x 128 lanes x 32 bit) ----------------------------------------
-constexpr uint32_t TM_S32 = 0;      // fp32 states S (dv x dk) of the item's one or two chains, 128 columns each
-constexpr uint32_t TM_SBF = 256;    // bf16 copy of the current step's start state, 64 columns
-constexpr uint32_t TM_ACC1 = 320;   // Delta^T accumulator (U^T - S0 W^T), 64 columns
-constexpr uint32_t TM_ACC2 = 384;   // O^T accumulator, 64 columns
-constexpr uint32_t TM_GRAM = 448;   // Gram accumulator, 64 columns
+constexpr uint32_t TM_S32 = 0;      // fp32 state S (dv x dk), 128 columns
+constexpr uint32_t TM_SBF = 128;    // bf16 copy of the chunk-start state, 64 columns
+constexpr uint32_t TM_ACC1 = 192;   // Delta^T accumulator (U^T - S0 W^T), 64 columns
+constexpr uint32_t TM_ACC2 = 256;   // S0 Q^T, 64 columns
+constexpr uint32_t TM_ACC3 = 320;   // Delta^T P^T, 64 columns
+constexpr uint32_t TM_GRAM = 384;   // Gram accumulator, 64 columns
+constexpr uint32_t TM_WACC = 448;   // W^T accumulator, 64 columns
 // The bf16 A operands Delta^T and Delta'^T replace the fp32 accumulator they are computed from, in place: the 16
 // fp32 columns of tokens [16 s, 16 s + 16) become 8 columns of Delta^T followed by 8 columns of Delta'^T.
 constexpr uint32_t TM_DBF = TM_ACC1;        // + 16 s
 constexpr uint32_t TM_DPBF = TM_ACC1 + 8;   // + 16 s
 
 constexpr uint32_t ID_GRAM = idesc_bf16(128, 64, 0, 0, 0);    // [K;Q] (K-major) x K (K-major)
-constexpr uint32_t ID_WU = idesc_bf16(128, 64, 1, 0, 0);      // V^T (M-major) x P^ (K-major)
+constexpr uint32_t ID_WU = idesc_bf16(128, 64, 1, 0, 0);      // K^T or V^T (M-major) x T (K-major)
 constexpr uint32_t ID_SW = idesc_bf16(128, 64, 0, 1, 1);      // -S0 (TMEM) x W^T (N-major)
 constexpr uint32_t ID_SQ = idesc_bf16(128, 64, 0, 0, 0);      // S0 (TMEM) x Q (K-major)
 constexpr uint32_t ID_DP = idesc_bf16(128, 64, 0, 0, 0);      // Delta^T (TMEM) x P (K-major)
@@ -127,71 +126,60 @@ struct TcParams {
     Problem p;
     Sched s;
     unsigned long long wait_timeout_ns;   // bound of every device-side wait
-    int32_t skip_kq_load;         // testing aid: index of the K/Q tile copy each CTA leaves out (-1: none)
-    int32_t ng;                   // chains per item: 1, or 2 (the two v-heads of a pair)
+    int32_t skip_kq_load;         // testing aid: chunk whose K/Q copy is left out (-1: none)
 };
 
-// Walks the step sequence of one CTA: items dealt in snake order over the longest-first request list, chunks of
-// 64 rows inside each item, the item's chains inside each chunk.  Every role keeps its own cursor(s).
-struct StepCursor {
+// Walks the chunk sequence of one CTA: chains dealt in snake order over the longest-first list,
+// chunks of 64 rows inside each chain.  Every role keeps its own cursor(s).
+struct ChunkCursor {
     const Problem* p;
     const int32_t* order;
-    int r, n, h0, hq, row_begin, row_end, nchunks, c, m, ng;
-    uint32_t num_items, u;            // u: running index of the (item, chunk) K/Q tile
+    int r, n, h, hq, row_begin, row_end, nchunks, c;
+    uint32_t num_items;
     bool valid;
 
-    __device__ void init(const TcParams& prm)
+    __device__ void init(const Problem* pp, const int32_t* ord)
     {
-        p = &prm.p; order = prm.s.order; ng = prm.ng; r = -1; c = 0; m = 0; nchunks = 0; u = 0; valid = true;
-        num_items = (uint32_t)p->num_seqs * (uint32_t)(p->Hv / ng);
-        next_item();
+        p = pp; order = ord; r = -1; c = 0; nchunks = 0; valid = true;
+        num_items = (uint32_t)pp->num_seqs * (uint32_t)pp->Hv;
+        next_chain();
     }
     __device__ static uint32_t item_of(int round)
     {
         const uint32_t G = gridDim.x, b = blockIdx.x;
         return (uint32_t)round * G + ((round & 1) ? (G - 1 - b) : b);
     }
-    // Row range and heads of one work item, kept out of line (integer divisions and two dependent global loads,
-    // needed once per item by every role): x = first row, y = end row, z = first v-head | q/k head << 16,
+    // Row range and heads of one work item, kept out of line (three integer divisions and two dependent
+    // global loads, needed once per chain by every role): x = first row, y = end row, z = v-head | q/k head << 16,
     // w = request index.
-    __device__ __noinline__ static int4 lookup(const Problem* p, const int32_t* order, uint32_t item, int ng)
+    __device__ __noinline__ static int4 lookup(const Problem* p, const int32_t* order, uint32_t item)
     {
-        const uint32_t per_req = (uint32_t)(p->Hv / ng);
-        const uint32_t slot = item / per_req;
-        const int n = order ? order[slot] : (int)slot;                         // no order list: requests as given
-        const int h0 = (int)(item % per_req) * ng;
-        const int hq = h0 / (p->Hv / p->Hq);
-        return make_int4(p->cu[n], p->cu[n + 1], h0 | (hq << 16), n);
+        const int n = order ? order[item / p->Hv] : (int)(item / p->Hv);       // no order list: requests as given
+        const int h = item % p->Hv;
+        const int hq = h / (p->Hv / p->Hq);
+        return make_int4(p->cu[n], p->cu[n + 1], h | (hq << 16), n);
     }
-    // moves to the next item that has at least one chunk
-    __device__ void next_item()
+    // moves to the next chain that has at least one chunk
+    __device__ void next_chain()
     {
         for (;;) {
             ++r;
             const uint32_t item = item_of(r);
             if (item >= num_items) { valid = false; return; }
-            const int4 ci = lookup(p, order, item, ng);
-            row_begin = ci.x; row_end = ci.y; h0 = ci.z & 0xffff; hq = ci.z >> 16; n = ci.w;
+            const int4 ci = lookup(p, order, item);
+            row_begin = ci.x; row_end = ci.y; h = ci.z & 0xffff; hq = ci.z >> 16; n = ci.w;
             nchunks = (row_end - row_begin + 63) >> 6;
-            c = 0; m = 0;
+            c = 0;
             if (nchunks > 0) return;
         }
     }
-    __device__ void advance()                 // next step
+    __device__ void advance()
     {
-        if (++m < ng) return;
-        next_kq();
+        if (++c >= nchunks) next_chain();
     }
-    __device__ void next_kq()                 // first step of the next (item, chunk)
-    {
-        m = 0; ++u;
-        if (++c >= nchunks) next_item();
-    }
-    __device__ int h() const { return h0 + m; }
     __device__ int row0() const { return row_begin + c * 64; }
     __device__ int nvalid() const { return min(64, row_end - row0()); }
     __device__ bool first() const { return c == 0; }
-    __device__ bool last() const { return c == nchunks - 1; }
 };
 
 struct Ctx {
@@ -202,8 +190,8 @@ struct Ctx {
     __device__ uint32_t bar(int i) const { return sb + SM_MISC + (uint32_t)offsetof(Misc, bars) + 8u * i; }
     __device__ bool stop() const { return __shfl_sync(0xffffffffu, misc->abort, 0) != 0u; }
     // Bounded wait.  On expiry it raises the CTA-wide abort flag; from then on no wait blocks any more, so
-    // every role still runs through its (data-independent) loop structure, keeps meeting its named barriers
-    // and reaches the end of the kernel; nothing more is stored and the host sees the status word.
+    // every role still runs through its (data-independent) loop structure, keeps meeting its warpgroup
+    // barriers and reaches the end of the kernel; the results are garbage and the host sees the status word.
     __device__ bool wait(int i, uint32_t parity) const
     {
         const uint32_t b = bar(i);
@@ -231,8 +219,13 @@ __device__ __forceinline__ void warp_arrive(uint32_t bar, int lane)
     __syncwarp();
     if (lane == 0) mbar_arrive(bar);
 }
-
-// ---- small bf16 tensor-core helpers (mma.sync with ldmatrix-fed fragments) ---------------------------
+// ---- small bf16 tensor-core helpers for the block merges of the triangular solve --------------------
+// Four 8x8 bf16 matrices of the 16 x 16 tile at (row0, col0) of a row-major shared-memory matrix:
+// plain -> A fragment {a0..a3}; transposed -> B fragments {b0, b1} of the two 8-column halves.
+__device__ __forceinline__ uint32_t tile_addr(uint32_t base, int ld, int row0, int col0, int lane)
+{
+    return base + (uint32_t)(((row0 + (lane & 7) + ((lane >> 3) & 1) * 8) * ld + col0 + (lane >> 4) * 8) * 2);
+}
 __device__ __forceinline__ void ldm_x4(uint32_t (&r)[4], uint32_t addr)
 {
     asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
@@ -243,27 +236,49 @@ __device__ __forceinline__ void ldm_x4_trans(uint32_t (&r)[4], uint32_t addr)
     asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
                  : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
 }
-__device__ __forceinline__ void ldm_x2_trans(uint32_t (&r)[2], uint32_t addr)
-{
-    asm volatile("ldmatrix.sync.aligned.m8n8.x2.trans.shared.b16 {%0,%1}, [%2];" : "=r"(r[0]), "=r"(r[1]) : "r"(addr));
-}
-__device__ __forceinline__ uint32_t ldm_x1(uint32_t addr)
-{
-    uint32_t r;
-    asm volatile("ldmatrix.sync.aligned.m8n8.x1.shared.b16 {%0}, [%1];" : "=r"(r) : "r"(addr));
-    return r;
-}
-__device__ __forceinline__ uint32_t ldm_x1_trans(uint32_t addr)
-{
-    uint32_t r;
-    asm volatile("ldmatrix.sync.aligned.m8n8.x1.trans.shared.b16 {%0}, [%1];" : "=r"(r) : "r"(addr));
-    return r;
-}
 __device__ __forceinline__ void mma_bf16(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1)
 {
     asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
                  : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
                  : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+// same four 8 x 8 matrices of a 64 x 64 bf16 tile kept in MMA operand layout: 128-byte rows, 16-byte chunk
+// index XORed with (row & 7)
+__device__ __forceinline__ uint32_t sw_off(int row, int col)
+{
+    return (uint32_t)(row * 128 + ((((col >> 3) ^ (row & 7))) << 4) + (col & 7) * 2);
+}
+__device__ __forceinline__ uint32_t tile_addr_sw(uint32_t base, int row0, int col0, int lane)
+{
+    return base + sw_off(row0 + (lane & 7) + ((lane >> 3) & 1) * 8, col0 + (lane >> 4) * 8);
+}
+// c (16 x 16, two 8-column halves) += A tile * B tile, each given by its per-lane ldmatrix address
+__device__ __forceinline__ void tile16_mma_at(float (&c)[2][4], uint32_t a_addr, uint32_t b_addr)
+{
+    uint32_t a[4], b[4];
+    ldm_x4(a, a_addr);
+    ldm_x4_trans(b, b_addr);
+    mma_bf16(c[0], a, b[0], b[1]);
+    mma_bf16(c[1], a, b[2], b[3]);
+}
+// stores sign * c as bf16 at D[r0.., n0..+16) (row-major, ld elements)
+__device__ __forceinline__ void tile16_store(const float (&c)[2][4], float sign, uint8_t* D, int ld, int r0, int n0, int lane)
+{
+    const int g = lane >> 2, t4 = lane & 3;
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+        *reinterpret_cast<uint32_t*>(D + ((r0 + g) * ld + n0 + 8 * h + 2 * t4) * 2) = pack_bf16x2(sign * c[h][0], sign * c[h][1]);
+        *reinterpret_cast<uint32_t*>(D + ((r0 + g + 8) * ld + n0 + 8 * h + 2 * t4) * 2) = pack_bf16x2(sign * c[h][2], sign * c[h][3]);
+    }
+}
+// 8 x 8 variants for the first merge level (two independent 8 x 8 problems per instruction pair)
+__device__ __forceinline__ void ldm_x2(uint32_t (&r)[2], uint32_t addr)
+{
+    asm volatile("ldmatrix.sync.aligned.m8n8.x2.shared.b16 {%0,%1}, [%2];" : "=r"(r[0]), "=r"(r[1]) : "r"(addr));
+}
+__device__ __forceinline__ void ldm_x2_trans(uint32_t (&r)[2], uint32_t addr)
+{
+    asm volatile("ldmatrix.sync.aligned.m8n8.x2.trans.shared.b16 {%0,%1}, [%2];" : "=r"(r[0]), "=r"(r[1]) : "r"(addr));
 }
 // rows 0-7 of (A[8 x 8] * B[8 x 8]) in c[0], c[1] (row lane / 4, columns 2 (lane % 4) + {0, 1})
 __device__ __forceinline__ void mma_8x8(float (&c)[4], uint32_t a0, uint32_t b0)
@@ -279,21 +294,6 @@ __device__ __forceinline__ uint32_t mul_bf16x2(uint32_t a, uint32_t b)
 }
 __device__ __forceinline__ float bf_lo(uint32_t w) { return __uint_as_float(w << 16); }
 __device__ __forceinline__ float bf_hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
-// element (row, col) of a 64-column bf16 tile kept in MMA operand layout: 128-byte rows, 16-byte chunk index
-// XORed with (row & 7) (the 128-byte swizzle of the TMA tiles and of the tcgen05 descriptors)
-__device__ __forceinline__ uint32_t sw_off(int row, int col)
-{
-    return (uint32_t)(row * 128 + ((((col >> 3) ^ (row & 7))) << 4) + (col & 7) * 2);
-}
-// per-lane ldmatrix.x4 address of the 16 x 16 tile at (row0, col0): matrices in the order
-// (rows 0-7, cols 0-7), (rows 8-15, cols 0-7), (rows 0-7, cols 8-15), (rows 8-15, cols 8-15)
-__device__ __forceinline__ uint32_t tile_addr_sw(uint32_t base, int row0, int col0, int lane)
-{
-    return base + sw_off(row0 + (lane & 7) + ((lane >> 3) & 1) * 8, col0 + (lane >> 4) * 8);
-}
-
-// advances the start-address field of a shared-memory descriptor by a byte offset
-__device__ __forceinline__ uint64_t desc_add(uint64_t d, uint32_t bytes) { return d + (uint64_t)(bytes >> 4); }
 
 // ================================================================================================
 // warp 0: TMA producer
@@ -301,12 +301,12 @@ __device__ __forceinline__ uint64_t desc_add(uint64_t d, uint32_t bytes) { retur
 __device__ void role_producer(const Ctx& cx, const TcParams& prm, const CUtensorMap* tm_q, const CUtensorMap* tm_k,
                               const CUtensorMap* tm_v)
 {
-    StepCursor ckq, cv;                  // K/Q runs two chunks ahead of V
-    ckq.init(prm);
+    ChunkCursor ckq, cv;                 // K/Q runs two chunks ahead of V
+    ckq.init(&prm.p, prm.s.order);
     cv = ckq;
-    auto load_kq = [&](const StepCursor& cc) {
-        const uint32_t slot = cc.u % 3u, dst = cx.sb + SM_KQ + slot * KQ_SLOT, bar = cx.bar(B_FULL_KQ0 + slot);
-        if ((int32_t)cc.u == prm.skip_kq_load) return;    // testing aid: this tile never arrives
+    auto load_kq = [&](const ChunkCursor& cc, uint32_t j) {
+        const uint32_t slot = j % NKQ, dst = cx.sb + SM_KQ + slot * KQ_SLOT, bar = cx.bar(B_FULL_KQ0 + slot);
+        if ((int32_t)j == prm.skip_kq_load) return;       // testing aid: this tile never arrives
         if (elect_one()) {
             mbar_arrive_expect_tx(bar, 32768u);
             tma_load_2d(dst, tm_k, cc.hq * 128, cc.row0(), bar);
@@ -316,43 +316,46 @@ __device__ void role_producer(const Ctx& cx, const TcParams& prm, const CUtensor
         }
         __syncwarp();
     };
-    for (int a = 0; a < 2 && ckq.valid; ++a) { load_kq(ckq); ckq.next_kq(); }
+    uint32_t jkq = 0;
+    for (; jkq < NKQ - 1 && ckq.valid; ++jkq) { load_kq(ckq, jkq); ckq.advance(); }
 #pragma unroll 1
-    for (uint32_t i = 0; cv.valid && !cx.stop(); ++i) {
-        // V(i): its slot held step i-2, free once the U^T MMA of that step has completed
-        const uint32_t vs = i & 1u;
-        if (i >= 2) cx.wait(B_V_FREE0 + vs, ((i >> 1) - 1u) & 1u);
-        const uint32_t bar = cx.bar(B_FULL_V0 + vs);
+    for (uint32_t j = 0; cv.valid && !cx.stop(); ++j) {
+        // V(j): the single slot is free once U^T MMA of chunk j-1 has completed
+        if (j >= 1) cx.wait(B_U_DONE, (j - 1) & 1u);
+        const uint32_t bar = cx.bar(B_FULL_V);
         if (elect_one()) {
             mbar_arrive_expect_tx(bar, 16384u);
-            tma_load_2d(cx.sb + SM_V + vs * V_SLOT, tm_v, cv.h() * 128, cv.row0(), bar);
-            tma_load_2d(cx.sb + SM_V + vs * V_SLOT + 8192, tm_v, cv.h() * 128 + 64, cv.row0(), bar);
+            tma_load_2d(cx.sb + SM_V, tm_v, cv.h * 128, cv.row0(), bar);
+            tma_load_2d(cx.sb + SM_V + 8192, tm_v, cv.h * 128 + 64, cv.row0(), bar);
         }
         __syncwarp();
-        // K/Q two chunks ahead: its slot held the chunk before this one, free once that chunk's last state
-        // update has completed
-        if (cv.m == 0 && ckq.valid) {
-            if (ckq.u >= 3) cx.wait(B_KQ_FREE0 + ckq.u % 3u, ((ckq.u / 3u) - 1u) & 1u);
-            load_kq(ckq);
-            ckq.next_kq();
-        }
         cv.advance();
+        // K/Q(j+2): its slot held chunk j-1, free once the state-update MMA of chunk j-1 has completed
+        if (ckq.valid) {
+            if (jkq >= NKQ) cx.wait(B_KQ_FREE0 + jkq % NKQ, ((jkq / NKQ) - 1u) & 1u);
+            load_kq(ckq, jkq);
+            ckq.advance();
+            ++jkq;
+        }
     }
 }
 
+// advances the start-address field of a shared-memory descriptor by a byte offset
+__device__ __forceinline__ uint64_t desc_add(uint64_t d, uint32_t bytes) { return d + (uint64_t)(bytes >> 4); }
+
 // ================================================================================================
-// warp 2: Gram MMAs, one per K/Q tile.  Needs the tile and the accumulator read by every step of the tile before.
+// warp 2: Gram MMAs.  Gram(j) needs the K/Q tiles of chunk j and the accumulator read by chunk j-1.
 // ================================================================================================
 __device__ void role_mma_gram(const Ctx& cx, const TcParams& prm)
 {
-    StepCursor cc;
-    cc.init(prm);
+    ChunkCursor cc;
+    cc.init(&prm.p, prm.s.order);
 #pragma unroll 1
-    for (; cc.valid; cc.next_kq()) {
-        const uint32_t u = cc.u, slot = u % 3u;
+    for (uint32_t j = 0; cc.valid; ++j, cc.advance()) {
+        const uint32_t slot = j % NKQ;
         const uint64_t d_kq = smem_desc_sw128(cx.sb + SM_KQ + slot * KQ_SLOT, 16, 1024);   // [K;Q] rows, K-major
-        cx.wait(B_FULL_KQ0 + slot, (u / 3u) & 1u);
-        if (u >= 1) cx.wait(B_GRAM_FREE, (u - 1) & 1u);
+        cx.wait(B_FULL_KQ0 + slot, (j / NKQ) & 1u);
+        if (j >= 1) cx.wait(B_GRAM_READ, (j - 1) & 1u);
         tc_fence_after();
         if (elect_one()) {
 #pragma unroll
@@ -360,9 +363,7 @@ __device__ void role_mma_gram(const Ctx& cx, const TcParams& prm)
                 const uint64_t d = desc_add(d_kq, (ks >> 2) * 16384 + (ks & 3) * 32);
                 mma_ss(cx.tmem + TM_GRAM, d, d, ID_GRAM, ks > 0);
             }
-            // one completion per step that reads this tile, on the barrier of the team that takes the step
-            mma_commit(cx.bar(B_GRAM_DONE0 + (u * (uint32_t)cc.ng) % 3u));
-            if (cc.ng == 2) mma_commit(cx.bar(B_GRAM_DONE0 + (u * 2u + 1u) % 3u));
+            mma_commit(cx.bar(B_GRAM_DONE));
         }
         __syncwarp();
     }
@@ -373,35 +374,36 @@ __device__ void role_mma_gram(const Ctx& cx, const TcParams& prm)
 // ================================================================================================
 __device__ void role_mma_chain(const Ctx& cx, const TcParams& prm)
 {
-    StepCursor cc;
-    cc.init(prm);
+    ChunkCursor cc;
+    cc.init(&prm.p, prm.s.order);
     const bool has_init = prm.p.init_state != nullptr;
+    const uint64_t d_v = smem_desc_sw128(cx.sb + SM_V, 8192, 1024);     // V tile as M-major operand (V^T)
     const uint64_t d_wt = smem_desc_sw128(cx.sb + SM_WT, 16, 1024);     // W^T rows [dk][t], N-major operand
 #pragma unroll 1
-    for (uint32_t i = 0; cc.valid; ++i, cc.advance()) {
-        const uint32_t kq = cx.sb + SM_KQ + (cc.u % 3u) * KQ_SLOT;
+    for (uint32_t j = 0; cc.valid; ++j, cc.advance()) {
+        const uint32_t kq = cx.sb + SM_KQ + (j % NKQ) * KQ_SLOT;
         const uint64_t d_q = smem_desc_sw128(kq + 8192, 16, 1024);      // Q rows, K-major
         const uint64_t d_kn = smem_desc_sw128(kq, 16384, 1024);         // K tile as N-major operand
-        const uint64_t d_v = smem_desc_sw128(cx.sb + SM_V + (i & 1u) * V_SLOT, 8192, 1024);   // V^T, M-major
-        const uint64_t d_p = smem_desc_sw128(cx.sb + SM_P + (i % RP) * 8192, 16, 1024);
-        const uint64_t d_tp = smem_desc_sw128(cx.sb + SM_TP + (i % RTP) * 8192, 16, 1024);
-        const uint32_t s32 = cx.tmem + TM_S32 + 128u * (uint32_t)cc.m;
-        const bool has_state = !cc.first() || has_init;
-        cx.wait(B_TP_READY0 + i % RTP, (i / RTP) & 1u);
-        cx.wait(B_FULL_V0 + (i & 1u), (i >> 1) & 1u);
+        const uint64_t d_p = smem_desc_sw128(cx.sb + SM_P + (j % 3u) * 8192, 16, 1024);
+        const uint64_t d_tp = smem_desc_sw128(cx.sb + SM_TP + (j % 3u) * 8192, 16, 1024);
+        const bool has_state = !cc.first() || has_init;     // a zero start state is skipped, not multiplied
+        cx.wait(B_TP_READY0 + j % 3u, (j / 3u) & 1u);
+        cx.wait(B_FULL_V, j & 1u);
         tc_fence_after();
-        // U^T = V^T P^^T -> ACC1 (free: the Delta operands of step i-1 in it were read by MMAs issued before
+        // U^T = V^T T'^T -> ACC1 (free: the Delta operands of chunk j-1 in it were read by MMAs issued before
         // these).  Issued ahead of the wait for the W^T operand, which is the last piece of the set to arrive.
         if (elect_one()) {
 #pragma unroll
             for (int ks = 0; ks < 4; ++ks)
                 mma_ss(cx.tmem + TM_ACC1, desc_add(d_v, ks * 2048), desc_add(d_tp, ks * 32), ID_WU, ks > 0);
-            mma_commit(cx.bar(B_V_FREE0 + (i & 1u)));
-            mma_commit(cx.bar(B_TP_FREE0 + i % RTP));
+            mma_commit(cx.bar(B_U_DONE));
+            mma_commit(cx.bar(B_TP_FREE0 + j % 3u));
         }
         __syncwarp();
-        cx.wait(B_PRE_DONE0 + i % 3u, (i / 3u) & 1u);
-        cx.wait(B_SBF_READY, i & 1u);
+        cx.wait(B_PRE_DONE0 + (j & 1u), (j >> 1) & 1u);
+        // start state of this chunk: the previous chunk's state converted, or, at a chain start, the previous chain's
+        // state read out and this chain's start state (if any) written
+        cx.wait(B_SBF_READY, j & 1u);
         tc_fence_after();
         if (has_state && elect_one()) {
 #pragma unroll
@@ -409,64 +411,58 @@ __device__ void role_mma_chain(const Ctx& cx, const TcParams& prm)
                 mma_ts(cx.tmem + TM_ACC1, cx.tmem + TM_SBF + ks * 8, desc_add(d_wt, ks * 2048), ID_SW, 1u);
         }
         __syncwarp();
-        // Delta^T is complete: its epilogue starts now, and the team of the next step may overwrite W^T
-        if (elect_one()) {
-            mma_commit(cx.bar(B_MMA1_DONE));
-            mma_commit(cx.bar(B_WT_FREE0 + (i + 1u) % 3u));
-        }
+        // Delta^T is complete: its epilogue starts now
+        if (elect_one()) mma_commit(cx.bar(B_MMA1_DONE));
         __syncwarp();
-        // S0 Q^T runs under the Delta epilogue; the output accumulator was released by the output group
-        if (i >= 1) cx.wait(B_ACC2_FREE, (i - 1) & 1u);
-        tc_fence_after();
-        if (has_state && elect_one()) {
-#pragma unroll
-            for (int ks = 0; ks < 8; ++ks)
-                mma_ts(cx.tmem + TM_ACC2, cx.tmem + TM_SBF + ks * 8,
-                       desc_add(d_q, (ks >> 2) * 16384 + (ks & 3) * 32), ID_SQ, ks > 0);
-        }
-        __syncwarp();
-        // the bf16 state has been read for the last time in this step
-        if (elect_one()) mma_commit(cx.bar(B_SQ_DONE));
-        __syncwarp();
-        cx.wait(B_D_READY, i & 1u);
+        // The state update only needs the Delta epilogue: it goes first, so that the chain never queues behind the
+        // output accumulators.
+        cx.wait(B_D_READY, j & 1u);
         tc_fence_after();
         if (elect_one()) {
 #pragma unroll
             for (int ks = 0; ks < 4; ++ks)
-                mma_ts(s32, cx.tmem + TM_DPBF + ks * 16, desc_add(d_kn, ks * 2048), ID_DK,
+                mma_ts(cx.tmem + TM_S32, cx.tmem + TM_DPBF + ks * 16, desc_add(d_kn, ks * 2048), ID_DK,
                        (has_state || ks > 0) ? 1u : 0u);
             mma_commit(cx.bar(B_STATE_DONE));
-            if (cc.m == cc.ng - 1) mma_commit(cx.bar(B_KQ_FREE0 + cc.u % 3u));     // K and Q of this chunk have been read
         }
         __syncwarp();
-        cx.wait(B_ACC2_SCALED, i & 1u);                     // S0 Q^T carries its e^G factors
+        // The two output products need the accumulators back from the output epilogue of chunk j-1.  S0 Q^T is the last
+        // reader of the bf16 state: the state epilogue waits for it (SQ_DONE) before it overwrites that copy.
+        if (j >= 1) cx.wait(B_ACC23_FREE, (j - 1) & 1u);
         tc_fence_after();
         if (elect_one()) {
+            if (has_state) {
+#pragma unroll
+                for (int ks = 0; ks < 8; ++ks)
+                    mma_ts(cx.tmem + TM_ACC2, cx.tmem + TM_SBF + ks * 8,
+                           desc_add(d_q, (ks >> 2) * 16384 + (ks & 3) * 32), ID_SQ, ks > 0);
+            }
+            mma_commit(cx.bar(B_SQ_DONE));
 #pragma unroll
             for (int ks = 0; ks < 4; ++ks)
-                mma_ts(cx.tmem + TM_ACC2, cx.tmem + TM_DBF + ks * 16, desc_add(d_p, ks * 32), ID_DP,
-                       (has_state || ks > 0) ? 1u : 0u);
+                mma_ts(cx.tmem + TM_ACC3, cx.tmem + TM_DBF + ks * 16, desc_add(d_p, ks * 32), ID_DP, ks > 0);
             mma_commit(cx.bar(B_MMA3_DONE));
-            mma_commit(cx.bar(B_P_FREE0 + i % RP));
+            mma_commit(cx.bar(B_P_FREE0 + j % 3u));
+            mma_commit(cx.bar(B_KQ_FREE0 + j % NKQ));           // K and Q of this chunk have been read
         }
         __syncwarp();
     }
 }
 
 // ================================================================================================
-// warp 3: decay warp.  Runs several steps ahead of the consumers (ring of RD slots), which hides the
+// warp 3: decay warp.  Runs up to three chunks ahead of the consumers (ring of four slots), which hides the
 // DRAM latency of the strided g / beta loads.
 // ================================================================================================
 __device__ void role_decay(const Ctx& cx, const TcParams& prm)
 {
     const Problem& p = prm.p;
     const int lane = threadIdx.x & 31;
-    StepCursor cc;
-    cc.init(prm);
-    float crun0 = 1.f, crun1 = 1.f;                           // running scale of each chain's stored state (see Decay)
+    ChunkCursor cc;
+    cc.init(&p, prm.s.order);
+    float c = 1.f;                                            // running scale of the stored state (see Decay)
 #pragma unroll 1
-    for (uint32_t i = 0; cc.valid; ++i, cc.advance()) {
-        const int row0 = cc.row0(), nvalid = cc.nvalid(), h = cc.h();
+    for (uint32_t j = 0; cc.valid; ++j, cc.advance()) {
+        const int row0 = cc.row0(), nvalid = cc.nvalid(), h = cc.h;
         const bool ok0 = lane < nvalid, ok1 = lane + 32 < nvalid;
         const float g0 = ok0 ? p.g[(size_t)(row0 + lane) * p.Hv + h] : 0.f;
         const float g1 = ok1 ? p.g[(size_t)(row0 + lane + 32) * p.Hv + h] : 0.f;
@@ -481,285 +477,355 @@ __device__ void role_decay(const Ctx& cx, const TcParams& prm)
         }
         G1 += __shfl_sync(0xffffffffu, G0, 31);
         const float GC = __shfl_sync(0xffffffffu, G1, 31);
-        const float crun = cc.m ? crun1 : crun0;
-        const float cprev = cc.first() ? 1.f : crun;
+        const float cprev = cc.first() ? 1.f : c;
         const float eGC = ex2_approx(GC);
         const bool rescale = cc.first() || !(cprev * eGC >= 9.094947e-13f);       // 2^-40; also catches NaN
-        const float c = rescale ? 1.f : cprev * eGC;
-        if (cc.m) crun1 = c; else crun0 = c;
+        c = rescale ? 1.f : cprev * eGC;
         const float cinv = rescale ? 1.f : __frcp_rn(c);
         const float e0 = ex2_approx(G0) * cprev, e1 = ex2_approx(G1) * cprev;
-        // the slot was last read by the chain and output groups in step i - RD
-        if (i >= RD) cx.wait(B_DECAY_FREE0 + (i % RD), ((i / RD) - 1u) & 1u);
-        Decay& dc = cx.misc->decay[i % RD];
-        dc.G2[lane] = G0; dc.G2[lane + 32] = G1;
+        // the slot was last read by the chain group's output epilogue of chunk j - 4
+        if (j >= 4) cx.wait(B_DECAY_FREE0 + (j & 3u), ((j >> 2) - 1u) & 1u);
+        Decay& dc = cx.misc->decay[j & 3u];
+        // rows past the end of the request (whose k, q, v may be anything finite) get a hugely negative cumulative
+        // decay: every Gam[t, .] of such a row underflows to zero, so its A^ and P rows vanish
+        dc.G2[lane] = ok0 ? G0 : -1.0e30f; dc.G2[lane + 32] = ok1 ? G1 : -1.0e30f;
         dc.beta[lane] = b0; dc.beta[lane + 32] = b1;
         dc.eG[lane] = e0; dc.eG[lane + 32] = e1;
         dc.bRest[lane] = b0 * (ex2_approx(GC - G0) * cinv); dc.bRest[lane + 32] = b1 * (ex2_approx(GC - G1) * cinv);
         const float G31 = __shfl_sync(0xffffffffu, G0, 31);
-        const float cf = ex2_approx(G31 - G0);
-        dc.colf[lane] = cf; dc.colfb[lane] = cf * b0;
-        if (lane == 0) { dc.wb = cprev * eGC; dc.G2mid = G31; dc.cfin = c; dc.rescale = rescale ? 1 : 0; dc.nvalid = nvalid; }
-        warp_arrive(cx.bar(B_DECAY_READY0 + (i % RD)), lane);
+        dc.colfb[lane] = ex2_approx(G31 - G0) * b0;
+        if (lane == 0) { dc.wb = cprev * eGC; dc.G2mid = G31; dc.cfin = c; dc.rescale = rescale ? 1 : 0; }
+        warp_arrive(cx.bar(B_DECAY_READY0 + (j & 3u)), lane);
+    }
+}
+
+// Number of 64-row chunks this CTA processes over all of its chains.
+__device__ __noinline__ uint32_t count_chunks(const TcParams& prm)
+{
+    ChunkCursor cc;
+    cc.init(&prm.p, prm.s.order);
+    uint32_t n = 0;
+    while (cc.valid) { n += (uint32_t)cc.nchunks; cc.next_chain(); }
+    return n;
+}
+
+// ================================================================================================
+// warps 4-11: group G1.  Per iteration k: Gram post-processing of chunk k+1 (writes A^ for the solve and the
+// operand P), then the W^T epilogue of chunk k.
+// ================================================================================================
+__device__ void role_g1(const Ctx& cx, const TcParams& prm, int wtid)
+{
+    const int lane = wtid & 31, pw = wtid >> 5;          // pw = 0..7
+    const int w4 = pw & 3, hf = pw >> 2;                 // TMEM lane window, column half
+    const uint32_t tl = cx.tmem + ((uint32_t)(w4 * 32) << 16);
+    Misc* misc = cx.misc;
+    const uint32_t J = count_chunks(prm);
+
+    // ---- Gram tile of chunk c -> A (bf16 scratch for the solve) and P (bf16 operand), 16 columns at a time
+    auto post = [&](uint32_t c) {
+        const Decay& dc = misc->decay[c & 3u];
+        cx.wait(B_DECAY_READY0 + (c & 3u), (c >> 2) & 1u);       // decay factors of this chunk are published
+        // this thread's row of the Gram tile: lane windows 0,1 hold K K^T rows, 2,3 hold Q K^T rows
+        const int t = ((w4 & 1) << 5) + lane;
+        const bool isA = w4 < 2;
+        const float G2t = dc.G2[t];
+        // the solve works on A^ = strict_lower(Gam (K K^T)) diag(beta) (beta on the columns): its inverse P^ gives
+        // T' = diag(beta) P^ and T'' = diag(beta) P^ diag(e^G), and the common row factor beta moves into the
+        // Delta epilogue, so that P^ itself is one MMA operand and its column-scaled copy the other
+        // (P carries beta on its columns as well, so that the output product takes Delta~ as it is)
+        const float* __restrict__ colscale = dc.beta;
+        const float* __restrict__ colfac = dc.colfb;
+        const int t_lim = isA ? t : t + 1;                      // keep columns s < t_lim
+        cx.wait(B_GRAM_DONE, c & 1u);
+        tc_fence_after();
+        // buffers: P and T' of chunk c were last read by the MMAs of chunk c-3
+        if (c >= 3) {
+            cx.wait(B_P_FREE0 + c % 3u, ((c / 3u) - 1u) & 1u);
+            cx.wait(B_TP_FREE0 + c % 3u, ((c / 3u) - 1u) & 1u);
+        }
+        // this thread's row of the operand tile it writes: A^ into T' (where the solve inverts it in place), or P
+        uint8_t* prow = cx.sm + (isA ? SM_TP : SM_P) + (c % 3u) * 8192 + t * 128;
+        // column blocks are dealt so that each warp of a lane window gets one block that touches the
+        // diagonal and one that does not: half 0 -> blocks {0, 2}, half 1 -> blocks {1, 3}
+        const bool lower_rows = (w4 & 1) != 0;                  // rows 32-63
+        const float rowf = lower_rows ? ex2_approx(G2t - dc.G2mid) : 0.f;
+#pragma unroll 1
+        for (int g = 0; g < 2; ++g) {
+            const int cb = hf + 2 * g, c0 = 16 * cb;
+            if (c0 > ((w4 & 1) << 5) + 31) {                    // block entirely above the diagonal (warp-uniform)
+                continue;                                       // (zero since the start of the kernel)
+            }
+            uint32_t acc[16];
+            tmem_ld16(tl + TM_GRAM + c0, acc);
+            tmem_ld_wait();
+            float vals[16];
+            if (lower_rows && cb < 2) {
+                // every column precedes every row of this warp: Gam = rowf * colf, no mask, no exp
+#pragma unroll
+                for (int i4 = 0; i4 < 4; ++i4) {
+                    const float4 cf = *reinterpret_cast<const float4*>(&colfac[c0 + 4 * i4]);
+                    vals[4 * i4 + 0] = (rowf * cf.x) * __uint_as_float(acc[4 * i4 + 0]);
+                    vals[4 * i4 + 1] = (rowf * cf.y) * __uint_as_float(acc[4 * i4 + 1]);
+                    vals[4 * i4 + 2] = (rowf * cf.z) * __uint_as_float(acc[4 * i4 + 2]);
+                    vals[4 * i4 + 3] = (rowf * cf.w) * __uint_as_float(acc[4 * i4 + 3]);
+                }
+            } else {
+#pragma unroll
+                for (int i4 = 0; i4 < 4; ++i4) {
+                    const float4 gs = *reinterpret_cast<const float4*>(&dc.G2[c0 + 4 * i4]);
+                    const float4 cs = *reinterpret_cast<const float4*>(&colscale[c0 + 4 * i4]);
+                    const float gss[4] = {gs.x, gs.y, gs.z, gs.w}, css[4] = {cs.x, cs.y, cs.z, cs.w};
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        const int i = 4 * i4 + e;
+                        // masked entries may overflow to inf / NaN before the select discards them
+                        const float f = ex2_approx(G2t - gss[e]) * css[e];
+                        vals[i] = (c0 + i < t_lim) ? f * __uint_as_float(acc[i]) : 0.f;
+                    }
+                }
+            }
+            uint4 u[2];
+#pragma unroll
+            for (int c8 = 0; c8 < 2; ++c8) {
+                u[c8].x = pack_bf16x2(vals[c8 * 8 + 0], vals[c8 * 8 + 1]);
+                u[c8].y = pack_bf16x2(vals[c8 * 8 + 2], vals[c8 * 8 + 3]);
+                u[c8].z = pack_bf16x2(vals[c8 * 8 + 4], vals[c8 * 8 + 5]);
+                u[c8].w = pack_bf16x2(vals[c8 * 8 + 6], vals[c8 * 8 + 7]);
+            }
+            *reinterpret_cast<uint4*>(prow + (((2 * cb) ^ (t & 7)) << 4)) = u[0];
+            *reinterpret_cast<uint4*>(prow + (((2 * cb + 1) ^ (t & 7)) << 4)) = u[1];
+        }
+        tc_fence_before();
+        warp_arrive(cx.bar(B_GRAM_READ), lane);                 // the accumulator may take the next Gram tile
+        fence_proxy_async_smem();                               // P is an MMA operand
+        // A^ of chunk c is complete: the solve may start.  (Barriers that follow a T' buffer are kept per buffer: the
+        // buffer's reuse then bounds how far an arrival can run ahead of a waiter, which a parity wait needs.)
+        warp_arrive(cx.bar(B_A_READY0 + c % 3u), lane);
+    };
+
+    // ---- W^T epilogue of chunk c: bf16 rows [dk][t] as the N-major operand of the S0 W^T MMA; completes the
+    // operand set of chunk c (each warp converts 32 columns of its lane window; TMEM lane = key index)
+    auto w_epilogue = [&](uint32_t c) {
+        cx.wait(B_W_DONE0 + (c & 1u), (c >> 1) & 1u);
+        tc_fence_after();
+        // W^T is single-buffered: the S0 W^T MMA of chunk c-1 must have read it
+        if (c >= 1) cx.wait(B_MMA1_DONE, (c - 1) & 1u);
+        const int drow = w4 * 32 + lane;
+        uint8_t* wrow = cx.sm + SM_WT + drow * 128;
+        const int c0 = 32 * hf;
+        uint32_t acc[32];
+        tmem_ld32(tl + TM_WACC + c0, acc);
+        tmem_ld_wait();
+#pragma unroll
+        for (int c8 = 0; c8 < 4; ++c8) {
+            uint4 u;
+            u.x = pack_bf16x2(__uint_as_float(acc[c8 * 8 + 0]), __uint_as_float(acc[c8 * 8 + 1]));
+            u.y = pack_bf16x2(__uint_as_float(acc[c8 * 8 + 2]), __uint_as_float(acc[c8 * 8 + 3]));
+            u.z = pack_bf16x2(__uint_as_float(acc[c8 * 8 + 4]), __uint_as_float(acc[c8 * 8 + 5]));
+            u.w = pack_bf16x2(__uint_as_float(acc[c8 * 8 + 6]), __uint_as_float(acc[c8 * 8 + 7]));
+            *reinterpret_cast<uint4*>(wrow + ((((c0 >> 3) + c8) ^ (drow & 7)) << 4)) = u;
+        }
+        tc_fence_before();
+        warp_arrive(cx.bar(B_WACC_READ), lane);                 // the accumulator may take the next W^T tile
+        fence_proxy_async_smem();
+        warp_arrive(cx.bar(B_PRE_DONE0 + (c & 1u)), lane);
+    };
+
+    // iteration i: Gram post-processing of chunk i, then the W^T epilogue of chunk i-1, whose solve and W^T MMA
+    // ran meanwhile
+#pragma unroll 1
+    for (uint32_t i = 0; i <= J; ++i) {
+        if (i < J) post(i);
+        if (i >= 1) w_epilogue(i - 1);
     }
 }
 
 // ================================================================================================
-// warps 4-15: pre-stage teams.  Team T (four warps, one per TMEM lane window) takes steps T, T + 3, ...:
-//   post   Gram tile -> A^ (into the step's P^ buffer) and P (operand), one thread per Gram row
-//   solve  P^ = (I + A^)^-1 in place.  Level 0: the eight 8 x 8 diagonal blocks by forward substitution in fp32;
-//          then 8 -> 16, 16 -> 32 and 32 -> 64 merges X[hi][lo] = -X[hi][hi] (A[hi][lo] X[lo][lo]) on mma.sync,
-//          every warp owning column tiles of the merged block so that no warp waits for another inside a level
-//   W      W~^T = K^T (P^ diag(e^G))^T on mma.sync, each warp 32 of the 128 key dimensions
+// warps 20-23: group G2 (two teams of two warps on alternate chunks), P^ = (I + A^)^-1 of chunk k.  Each warp of a
+// team inverts one 32 x 32 diagonal half without any cross-warp barrier:
+//   level 0  : its four 8 x 8 diagonal blocks by forward substitution in fp32
+//   level 0.5: 8 -> 16 merges, level 1: the 16 -> 32 merge X[hi][lo] = -X[hi][hi] (A[hi][lo] X[lo][lo]),
+//   level 2  : X[32:64][0:32] = -X22 (A21 X11), two 16 x 16 tiles per warp,
+// the merges on mma.sync with ldmatrix-fed bf16 fragments.  The post-processing has left A^ in the chunk's T' operand
+// buffer (MMA operand layout, which ldmatrix reads just as well), and the inverse replaces it block by block: every
+// block is read by the warp that overwrites it, before it does.  A last pass writes the copy with columns scaled by
+// e^G into the T'' operand buffer.  What lies above the 16 x 16 diagonal blocks of both is zero from the start of
+// the kernel.
 // ================================================================================================
-__device__ void role_team(const Ctx& cx, const TcParams& prm, int team, int tw, int lane)
+// stores sign * c of a 16 x 16 accumulator tile (two 8-column halves) at rows r0.., columns n0.. of an operand tile
+__device__ __forceinline__ void tile16_store_sw(const float (&c)[2][4], float sign, uint8_t* T, int r0, int n0, int lane)
 {
-    Misc* misc = cx.misc;
-    const uint32_t tl = cx.tmem + ((uint32_t)(tw * 32) << 16);
-    const uint32_t mhw = cx.sb + SM_MH + (uint32_t)(team * 4 + tw) * 512u;      // this warp's merge scratch
-    uint8_t* MHW = cx.sm + SM_MH + (team * 4 + tw) * 512;
-    auto team_sync = [&]() { asm volatile("bar.sync %0, 128;" ::"r"(2 + team) : "memory"); };
     const int g = lane >> 2, t4 = lane & 3;
-    StepCursor cc;
-    cc.init(prm);
-    for (int a = 0; a < team && cc.valid; ++a) cc.advance();
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+        *reinterpret_cast<uint32_t*>(T + sw_off(r0 + g, n0 + 8 * h + 2 * t4)) = pack_bf16x2(sign * c[h][0], sign * c[h][1]);
+        *reinterpret_cast<uint32_t*>(T + sw_off(r0 + g + 8, n0 + 8 * h + 2 * t4)) = pack_bf16x2(sign * c[h][2], sign * c[h][3]);
+    }
+}
+
+__device__ void role_g2(const Ctx& cx, const TcParams& prm, int wtid, int team)
+{
+    const int lane = wtid & 31, pw = wtid >> 5;          // pw = 0, 1
+    uint8_t* MH = cx.sm + SM_MH + team * MH_BYTES;
+    const uint32_t mh = cx.sb + SM_MH + team * MH_BYTES;
+    const uint32_t J = count_chunks(prm);
+    auto pair_sync = [&]() { asm volatile("bar.sync %0, 64;" ::"r"(3 + team) : "memory"); };
+    // team 0 takes the even chunks, team 1 the odd ones: the A, T' and T'' buffers alternate the same way
 #pragma unroll 1
-    for (uint32_t i = (uint32_t)team; cc.valid; i += kTeams) {
-        const uint32_t u = cc.u;
-        const uint32_t kq = cx.sb + SM_KQ + (u % 3u) * KQ_SLOT;
-        const Decay& dc = misc->decay[i % RD];
-        uint8_t* TP = cx.sm + SM_TP + (i % RTP) * 8192;
-        const uint32_t xs = cx.sb + SM_TP + (i % RTP) * 8192;
-        cx.wait(B_DECAY_READY0 + (i % RD), (i / RD) & 1u);
-        // buffers of this step: P^ was last read by the U^T MMA of step i - RTP, P by the MMAs of step i - RP
-        if (i >= RTP) cx.wait(B_TP_FREE0 + i % RTP, ((i / RTP) - 1u) & 1u);
-        if (i >= RP) cx.wait(B_P_FREE0 + i % RP, ((i / RP) - 1u) & 1u);
-        cx.wait(B_FULL_KQ0 + u % 3u, (u / 3u) & 1u);
-        cx.wait(B_GRAM_DONE0 + team, (i / 3u) & 1u);
-        tc_fence_after();
-        // ---- post: this thread's row of the Gram tile; lane windows 0,1 hold K K^T rows, 2,3 hold Q K^T rows ----
+    for (uint32_t k = (uint32_t)team; k < J; k += 2) {
+        cx.wait(B_A_READY0 + k % 3u, (k / 3u) & 1u);
+        const Decay& dc = cx.misc->decay[k & 3u];
+        uint8_t* TP = cx.sm + SM_TP + (k % 3u) * 8192;           // holds A^; becomes the inverse
+        const uint32_t xs = cx.sb + SM_TP + (k % 3u) * 8192;
         {
-            const int t = ((tw & 1) << 5) + lane;
-            const bool isA = tw < 2;
-            const float G2t = dc.G2[t];
-            const float* __restrict__ colscale = isA ? dc.beta : misc->ones;
-            const float* __restrict__ colfac = isA ? dc.colfb : dc.colf;
-            // keep columns s < t_lim; rows past the end of the request (whose k, q may be anything) are zeroed
-            const bool row_ok = t < dc.nvalid;
-            const int t_lim = row_ok ? (isA ? t : t + 1) : 0;
-            uint8_t* orow = (isA ? TP : cx.sm + SM_P + (i % RP) * 8192) + t * 128;
-            const bool lower_rows = (tw & 1) != 0;                  // rows 32-63
-            const float rowf = (lower_rows && row_ok) ? ex2_approx(G2t - dc.G2mid) : 0.f;
-            const int nblk = lower_rows ? 4 : 2;                    // 16-column blocks that reach the diagonal
-#pragma unroll 1
-            for (int cb = 0; cb < nblk; ++cb) {
-                const int c0 = 16 * cb;
-                uint32_t acc[16];
-                tmem_ld16(tl + TM_GRAM + c0, acc);
-                tmem_ld_wait();
-                float vals[16];
-                if (lower_rows && cb < 2) {
-                    // every column precedes every row of this warp: Gam = rowf * colf, no mask, no exp
-#pragma unroll
-                    for (int i4 = 0; i4 < 4; ++i4) {
-                        const float4 cf = *reinterpret_cast<const float4*>(&colfac[c0 + 4 * i4]);
-                        vals[4 * i4 + 0] = (rowf * cf.x) * __uint_as_float(acc[4 * i4 + 0]);
-                        vals[4 * i4 + 1] = (rowf * cf.y) * __uint_as_float(acc[4 * i4 + 1]);
-                        vals[4 * i4 + 2] = (rowf * cf.z) * __uint_as_float(acc[4 * i4 + 2]);
-                        vals[4 * i4 + 3] = (rowf * cf.w) * __uint_as_float(acc[4 * i4 + 3]);
-                    }
-                } else {
-#pragma unroll
-                    for (int i4 = 0; i4 < 4; ++i4) {
-                        const float4 gs = *reinterpret_cast<const float4*>(&dc.G2[c0 + 4 * i4]);
-                        const float4 cs = *reinterpret_cast<const float4*>(&colscale[c0 + 4 * i4]);
-                        const float gss[4] = {gs.x, gs.y, gs.z, gs.w}, css[4] = {cs.x, cs.y, cs.z, cs.w};
-#pragma unroll
-                        for (int e = 0; e < 4; ++e) {
-                            const int ii = 4 * i4 + e;
-                            // masked entries may overflow to inf / NaN before the select discards them
-                            const float f = ex2_approx(G2t - gss[e]) * css[e];
-                            vals[ii] = (c0 + ii < t_lim) ? f * __uint_as_float(acc[ii]) : 0.f;
-                        }
-                    }
-                }
-                uint4 v0, v1;
-                v0.x = pack_bf16x2(vals[0], vals[1]); v0.y = pack_bf16x2(vals[2], vals[3]);
-                v0.z = pack_bf16x2(vals[4], vals[5]); v0.w = pack_bf16x2(vals[6], vals[7]);
-                v1.x = pack_bf16x2(vals[8], vals[9]); v1.y = pack_bf16x2(vals[10], vals[11]);
-                v1.z = pack_bf16x2(vals[12], vals[13]); v1.w = pack_bf16x2(vals[14], vals[15]);
-                *reinterpret_cast<uint4*>(orow + (((2 * cb) ^ (t & 7)) << 4)) = v0;
-                *reinterpret_cast<uint4*>(orow + (((2 * cb + 1) ^ (t & 7)) << 4)) = v1;
-            }
-            tc_fence_before();
-            warp_arrive(cx.bar(B_GRAM_FREE), lane);             // this step is done with the Gram accumulator
-        }
-        team_sync();                                            // A^ is complete
-        // ---- solve, in place in the P^ buffer ------------------------------------------------------------------
-        // level 0: diagonal 8 x 8 blocks 2 tw and 2 tw + 1, one thread per column (lanes 0-15)
-        {
-            const int b = 8 * (2 * tw + ((lane >> 3) & 1)), jj = lane & 7;
+            const int bb = 4 * pw + (lane >> 3), b = 8 * bb, jj = lane & 7;
             uint4 rows[7];
 #pragma unroll
             for (int r = 1; r < 8; ++r) rows[r - 1] = *reinterpret_cast<const uint4*>(TP + sw_off(b + r, b));
             __syncwarp();                                       // every row is in registers before any is overwritten
-            if (lane < 16) {
-                float x[8];
+            float x[8];
 #pragma unroll
-                for (int r = 0; r < 8; ++r) x[r] = (r == jj) ? 1.f : 0.f;
+            for (int r = 0; r < 8; ++r) x[r] = (r == jj) ? 1.f : 0.f;
 #pragma unroll
-                for (int r = 1; r < 8; ++r) {
-                    const uint32_t wds[4] = {rows[r - 1].x, rows[r - 1].y, rows[r - 1].z, rows[r - 1].w};
-                    float acc0 = 0.f, acc1 = 0.f;
+            for (int r = 1; r < 8; ++r) {
+                const uint32_t wds[4] = {rows[r - 1].x, rows[r - 1].y, rows[r - 1].z, rows[r - 1].w};
+                float acc0 = 0.f, acc1 = 0.f;
 #pragma unroll
-                    for (int s2 = 0; s2 < r; ++s2) {
-                        const float a = (s2 & 1) ? bf_hi(wds[s2 >> 1]) : bf_lo(wds[s2 >> 1]);
-                        if (s2 & 1) acc1 = fmaf(a, x[s2], acc1); else acc0 = fmaf(a, x[s2], acc0);
-                    }
-                    x[r] = (r > jj) ? -(acc0 + acc1) : x[r];
+                for (int s2 = 0; s2 < r; ++s2) {
+                    const float a = (s2 & 1) ? bf_hi(wds[s2 >> 1]) : bf_lo(wds[s2 >> 1]);
+                    if (s2 & 1) acc1 = fmaf(a, x[s2], acc1); else acc0 = fmaf(a, x[s2], acc0);
                 }
-                // this thread's column of the diagonal block, zeros above the diagonal included
-#pragma unroll
-                for (int r = 0; r < 8; ++r)
-                    *reinterpret_cast<__nv_bfloat16*>(TP + sw_off(b + r, b + jj)) = __float2bfloat16_rn(x[r]);
+                x[r] = (r > jj) ? -(acc0 + acc1) : x[r];
             }
+            // this thread's column of the diagonal block, zeros above the diagonal included
+#pragma unroll
+            for (int r = 0; r < 8; ++r)
+                *reinterpret_cast<__nv_bfloat16*>(TP + sw_off(b + r, b + jj)) = __float2bfloat16_rn(x[r]);
         }
         __syncwarp();
-        // 8 -> 16 merge of diagonal block tw
         {
-            const int b16 = 16 * tw, rr = lane & 7;
-            const uint32_t a21 = ldm_x1(xs + sw_off(b16 + 8 + rr, b16));
-            const uint32_t x11 = ldm_x1_trans(xs + sw_off(b16 + rr, b16));
-            float m0[4] = {0.f, 0.f, 0.f, 0.f};
-            mma_8x8(m0, a21, x11);
-            *reinterpret_cast<uint32_t*>(MHW + g * 16 + t4 * 4) = pack_bf16x2(m0[0], m0[1]);
+            const int i = (lane >> 3) & 1, rr = lane & 7, b16 = 32 * pw + 16 * i;
+            const int g = lane >> 2, t4 = lane & 3;
+            uint32_t a[2], bx[2];
+            ldm_x2(a, xs + sw_off(b16 + 8 + rr, b16));                            // A21 of both blocks
+            ldm_x2_trans(bx, xs + sw_off(b16 + rr, b16));                         // X11 of both blocks
+            float m0[4] = {0.f, 0.f, 0.f, 0.f}, m1[4] = {0.f, 0.f, 0.f, 0.f};
+            mma_8x8(m0, a[0], bx[0]);
+            mma_8x8(m1, a[1], bx[1]);
+            *reinterpret_cast<uint32_t*>(MH + ((16 * pw + g) * LDM + 2 * t4) * 2) = pack_bf16x2(m0[0], m0[1]);
+            *reinterpret_cast<uint32_t*>(MH + ((16 * pw + 8 + g) * LDM + 2 * t4) * 2) = pack_bf16x2(m1[0], m1[1]);
             __syncwarp();
-            const uint32_t x22 = ldm_x1(xs + sw_off(b16 + 8 + rr, b16 + 8));
-            const uint32_t mm = ldm_x1_trans(mhw + rr * 16);
-            float d0[4] = {0.f, 0.f, 0.f, 0.f};
-            mma_8x8(d0, x22, mm);
-            *reinterpret_cast<uint32_t*>(TP + sw_off(b16 + 8 + g, b16 + 2 * t4)) = pack_bf16x2(-d0[0], -d0[1]);
+            uint32_t a2[2], bm[2];
+            ldm_x2(a2, xs + sw_off(b16 + 8 + rr, b16 + 8));                       // X22 of both blocks
+            ldm_x2_trans(bm, mh + ((16 * pw + 8 * i + rr) * LDM) * 2);           // M of both blocks
+            float d0[4] = {0.f, 0.f, 0.f, 0.f}, d1[4] = {0.f, 0.f, 0.f, 0.f};
+            mma_8x8(d0, a2[0], bm[0]);
+            mma_8x8(d1, a2[1], bm[1]);
+            const int c0b = 32 * pw, c1b = 32 * pw + 16;
+            *reinterpret_cast<uint32_t*>(TP + sw_off(c0b + 8 + g, c0b + 2 * t4)) = pack_bf16x2(-d0[0], -d0[1]);
+            *reinterpret_cast<uint32_t*>(TP + sw_off(c1b + 8 + g, c1b + 2 * t4)) = pack_bf16x2(-d1[0], -d1[1]);
         }
-        // 16 -> 32 merge of diagonal half tw / 2: this warp owns 8 of the 16 columns.  The A block is taken into
-        // registers before the team meets, i.e. before the other warp of the half overwrites its columns of it.
-        const int lo = 32 * (tw >> 1), hi = lo + 16, nh = tw & 1;
-        uint32_t aL1[4];
-        ldm_x4(aL1, tile_addr_sw(xs, hi, lo, lane));
-        team_sync();                                            // all 16 x 16 diagonal blocks are inverted
-        // the A operands of the last merge, likewise taken before anybody writes the block
-        uint32_t aL2[2][2][4];
-#pragma unroll
-        for (int mb = 0; mb < 2; ++mb)
-#pragma unroll
-            for (int kb = 0; kb < 2; ++kb) ldm_x4(aL2[mb][kb], tile_addr_sw(xs, 32 + 16 * mb, 16 * kb, lane));
+        __syncwarp();
         {
-            uint32_t bx[2];
-            ldm_x2_trans(bx, xs + sw_off(lo + (lane & 15), lo + 8 * nh));            // X[lo][lo], columns of this warp
-            float mt[4] = {0.f, 0.f, 0.f, 0.f};
-            mma_bf16(mt, aL1, bx[0], bx[1]);
-            *reinterpret_cast<uint32_t*>(MHW + g * 16 + t4 * 4) = pack_bf16x2(mt[0], mt[1]);
-            *reinterpret_cast<uint32_t*>(MHW + (g + 8) * 16 + t4 * 4) = pack_bf16x2(mt[2], mt[3]);
-            __syncwarp();
-            uint32_t a2[4], bm[2];
-            ldm_x4(a2, tile_addr_sw(xs, hi, hi, lane));                               // X[hi][hi]
-            ldm_x2_trans(bm, mhw + (lane & 15) * 16);
-            float d[4] = {0.f, 0.f, 0.f, 0.f};
-            mma_bf16(d, a2, bm[0], bm[1]);
-            *reinterpret_cast<uint32_t*>(TP + sw_off(hi + g, lo + 8 * nh + 2 * t4)) = pack_bf16x2(-d[0], -d[1]);
-            *reinterpret_cast<uint32_t*>(TP + sw_off(hi + g + 8, lo + 8 * nh + 2 * t4)) = pack_bf16x2(-d[2], -d[3]);
-        }
-        team_sync();                                            // both 32 x 32 diagonal halves are inverted
-        // 32 -> 64 merge: X[32:64][0:32] = -X22 (A21 X11); this warp owns columns [8 tw, 8 tw + 8)
-        {
-            float mt[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
-#pragma unroll
-            for (int kb = 0; kb < 2; ++kb) {
-                if (kb == 0 && tw >= 2) continue;               // X11 is lower triangular: rows 0-15 have no entry in columns 16-31
-                uint32_t bx[2];
-                ldm_x2_trans(bx, xs + sw_off(16 * kb + (lane & 15), 8 * tw));
-                mma_bf16(mt[0], aL2[0][kb], bx[0], bx[1]);
-                mma_bf16(mt[1], aL2[1][kb], bx[0], bx[1]);
-            }
-#pragma unroll
-            for (int mb = 0; mb < 2; ++mb) {
-                *reinterpret_cast<uint32_t*>(MHW + (16 * mb + g) * 16 + t4 * 4) = pack_bf16x2(mt[mb][0], mt[mb][1]);
-                *reinterpret_cast<uint32_t*>(MHW + (16 * mb + g + 8) * 16 + t4 * 4) = pack_bf16x2(mt[mb][2], mt[mb][3]);
-            }
+            const int lo = 32 * pw, hi = 32 * pw + 16;
+            float m[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
+            tile16_mma_at(m, tile_addr_sw(xs, hi, lo, lane), tile_addr_sw(xs, lo, lo, lane));          // A[hi][lo] X[lo][lo]
+            tile16_store(m, 1.f, MH, LDM, 16 * pw, 0, lane);
             __syncwarp();
             float d[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
-            uint32_t bm[2][2];
-            ldm_x2_trans(bm[0], mhw + (lane & 15) * 16);
-            ldm_x2_trans(bm[1], mhw + (16 + (lane & 15)) * 16);
-            uint32_t a2[4];
-            ldm_x4(a2, tile_addr_sw(xs, 32, 32, lane));                               // X22 is lower triangular
-            mma_bf16(d[0], a2, bm[0][0], bm[0][1]);
-            ldm_x4(a2, tile_addr_sw(xs, 48, 32, lane));
-            mma_bf16(d[1], a2, bm[0][0], bm[0][1]);
-            ldm_x4(a2, tile_addr_sw(xs, 48, 48, lane));
-            mma_bf16(d[1], a2, bm[1][0], bm[1][1]);
-#pragma unroll
-            for (int mb = 0; mb < 2; ++mb) {
-                *reinterpret_cast<uint32_t*>(TP + sw_off(32 + 16 * mb + g, 8 * tw + 2 * t4)) = pack_bf16x2(-d[mb][0], -d[mb][1]);
-                *reinterpret_cast<uint32_t*>(TP + sw_off(32 + 16 * mb + g + 8, 8 * tw + 2 * t4)) = pack_bf16x2(-d[mb][2], -d[mb][3]);
+            tile16_mma_at(d, tile_addr_sw(xs, hi, hi, lane), tile_addr(mh, LDM, 16 * pw, 0, lane));   // X[hi][hi] M
+            tile16_store_sw(d, -1.f, TP, hi, lo, lane);
+        }
+        pair_sync();
+        // level 2: warp pw owns block row mt = pw of X[32:64][0:32] (it alone reads and then overwrites those rows);
+        // its two 16 x 16 tiles are independent, so their ldmatrix / mma chains are written side by side
+        {
+            const int mt = pw;
+            float m0[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}}, m1[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
+            // X11 is lower triangular: block column nt starts at block row nt
+            tile16_mma_at(m0, tile_addr_sw(xs, 32 + 16 * mt, 0, lane), tile_addr_sw(xs, 0, 0, lane));
+            tile16_mma_at(m1, tile_addr_sw(xs, 32 + 16 * mt, 16, lane), tile_addr_sw(xs, 16, 16, lane));
+            tile16_mma_at(m0, tile_addr_sw(xs, 32 + 16 * mt, 16, lane), tile_addr_sw(xs, 16, 0, lane));
+            tile16_store(m0, 1.f, MH, LDM, 16 * mt, 0, lane);
+            tile16_store(m1, 1.f, MH, LDM, 16 * mt, 16, lane);
+            pair_sync();
+            float d0[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}}, d1[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
+            // X22 is lower triangular: block row mt ends at block column mt
+            tile16_mma_at(d0, tile_addr_sw(xs, 32 + 16 * mt, 32, lane), tile_addr(mh, LDM, 0, 0, lane));
+            tile16_mma_at(d1, tile_addr_sw(xs, 32 + 16 * mt, 32, lane), tile_addr(mh, LDM, 0, 16, lane));
+            if (mt == 1) {
+                tile16_mma_at(d0, tile_addr_sw(xs, 48, 48, lane), tile_addr(mh, LDM, 16, 0, lane));
+                tile16_mma_at(d1, tile_addr_sw(xs, 48, 48, lane), tile_addr(mh, LDM, 16, 16, lane));
             }
+            tile16_store_sw(d0, -1.f, TP, 32 + 16 * mt, 0, lane);
+            tile16_store_sw(d1, -1.f, TP, 32 + 16 * mt, 16, lane);
         }
-        fence_proxy_async_smem();                               // P^ (and P) are MMA operands
-        warp_arrive(cx.bar(B_TP_READY0 + i % RTP), lane);
-        team_sync();                                            // the whole of P^ is in place
-        // ---- W~^T = K^T (P^ diag(e^G))^T: this warp computes key dimensions [32 tw, 32 tw + 32) ----------------
-        uint32_t esc[4][2];                                     // e^G of the tokens this lane's A fragments cover
-#pragma unroll
-        for (int ks = 0; ks < 4; ++ks) {
-            const float2 ea = *reinterpret_cast<const float2*>(&dc.eG[16 * ks + 2 * t4]);
-            const float2 eb = *reinterpret_cast<const float2*>(&dc.eG[16 * ks + 8 + 2 * t4]);
-            esc[ks][0] = pack_bf16x2(ea.x, ea.y);
-            esc[ks][1] = pack_bf16x2(eb.x, eb.y);
-        }
-        // W^T is single-buffered: the S0 W^T MMA of step i-1 must have read it (its completion is this team's
-        // (i / 3)-th, for team 0, whose step 0 has no predecessor, (i / 3 - 1)-th)
-        if (i >= 1) cx.wait(B_WT_FREE0 + team, ((i / 3u) - (team == 0 ? 1u : 0u)) & 1u);
+        fence_proxy_async_smem();                               // T' is an MMA operand
+        warp_arrive(cx.bar(B_TP_READY0 + k % 3u), lane);
+        pair_sync();                                            // the whole inverse is in place
+        // T'' = T' diag(e^G): this thread's row, 16-byte chunks up to the diagonal.  The one T'' buffer was last read by
+        // the W^T MMA of chunk k-1 (the other team's; consecutive phases of its barrier are observed chunk after chunk).
+        if (k >= 1) cx.wait(B_W_DONE0 + ((k - 1) & 1u), ((k - 1) >> 1) & 1u);
+        {
+            const int t = 32 * pw + lane;
+            const uint8_t* src = TP + t * 128;
+            uint8_t* dst = cx.sm + SM_TPP + t * 128;
 #pragma unroll 1
-        for (int dbl = 0; dbl < 2; ++dbl) {
-            const int d0 = 32 * tw + 16 * dbl;                  // 16 key dimensions
-            float acc[8][4];
-#pragma unroll
-            for (int nt = 0; nt < 8; ++nt) { acc[nt][0] = acc[nt][1] = acc[nt][2] = acc[nt][3] = 0.f; }
-            const uint32_t kbase = kq + (uint32_t)(d0 >> 6) * 16384u;
-            const int dchunk = ((d0 & 63) >> 3) + ((lane >> 3) & 1);
-#pragma unroll
-            for (int ks = 0; ks < 4; ++ks) {
-                // (K^T) fragment: tokens 16 ks .. +15 (rows of the K tile), transposed on the way in
-                const int srow = 16 * ks + (lane & 7) + ((lane >> 4) & 1) * 8;
-                uint32_t a[4];
-                ldm_x4_trans(a, kbase + (uint32_t)(srow * 128 + ((dchunk ^ (srow & 7)) << 4)));
-                a[0] = mul_bf16x2(a[0], esc[ks][0]); a[1] = mul_bf16x2(a[1], esc[ks][0]);
-                a[2] = mul_bf16x2(a[2], esc[ks][1]); a[3] = mul_bf16x2(a[3], esc[ks][1]);
-                // P^ is lower triangular: token block nb >= ks only
-#pragma unroll
-                for (int nb = ks; nb < 4; ++nb) {
-                    uint32_t b[4];
-                    ldm_x4(b, tile_addr_sw(xs, 16 * nb, 16 * ks, lane));
-                    mma_bf16(acc[2 * nb], a, b[0], b[2]);
-                    mma_bf16(acc[2 * nb + 1], a, b[1], b[3]);
-                }
-            }
-            uint8_t* WT = cx.sm + SM_WT;
-#pragma unroll
-            for (int nt = 0; nt < 8; ++nt) {
-                *reinterpret_cast<uint32_t*>(WT + sw_off(d0 + g, 8 * nt + 2 * t4)) = pack_bf16x2(acc[nt][0], acc[nt][1]);
-                *reinterpret_cast<uint32_t*>(WT + sw_off(d0 + g + 8, 8 * nt + 2 * t4)) = pack_bf16x2(acc[nt][2], acc[nt][3]);
+            for (int ch = 0; ch <= (t >> 3); ++ch) {
+                const uint4 v = *reinterpret_cast<const uint4*>(src + ((ch ^ (t & 7)) << 4));
+                const float4 e0 = *reinterpret_cast<const float4*>(&dc.eG[8 * ch]);
+                const float4 e1 = *reinterpret_cast<const float4*>(&dc.eG[8 * ch + 4]);
+                uint4 o;
+                o.x = mul_bf16x2(v.x, pack_bf16x2(e0.x, e0.y)); o.y = mul_bf16x2(v.y, pack_bf16x2(e0.z, e0.w));
+                o.z = mul_bf16x2(v.z, pack_bf16x2(e1.x, e1.y)); o.w = mul_bf16x2(v.w, pack_bf16x2(e1.z, e1.w));
+                *reinterpret_cast<uint4*>(dst + ((ch ^ (t & 7)) << 4)) = o;
             }
         }
-        fence_proxy_async_smem();
-        warp_arrive(cx.bar(B_PRE_DONE0 + team), lane);
-        cc.advance();
-        if (cc.valid) cc.advance();
-        if (cc.valid) cc.advance();
+        fence_proxy_async_smem();                               // T'' is an MMA operand
+        pair_sync();                                            // both warps' rows of T'' are in place
+        // W~^T = K^T T''^T, issued from here: needs the accumulator read by the W^T epilogue of chunk k-1
+        if (pw == 0) {
+            const uint64_t d_kt = smem_desc_sw128(cx.sb + SM_KQ + (k % NKQ) * KQ_SLOT, 16384, 1024);   // K^T, M-major
+            const uint64_t d_tpp = smem_desc_sw128(cx.sb + SM_TPP, 16, 1024);
+            if (k >= 1) cx.wait(B_WACC_READ, (k - 1) & 1u);
+            tc_fence_after();
+            if (elect_one()) {
+#pragma unroll
+                for (int ks = 0; ks < 4; ++ks)
+                    mma_ss(cx.tmem + TM_WACC, desc_add(d_kt, ks * 2048), desc_add(d_tpp, ks * 32), ID_WU, ks > 0);
+                mma_commit(cx.bar(B_W_DONE0 + (k & 1u)));
+            }
+            __syncwarp();
+        }
     }
 }
 
+// Start state of a chain from init_state [dk][dv] fp32 (kept out of line: most calls start from zero).  The first chunk
+// starts from a rescaled state (see Decay): the fp32 copy is multiplied by wb of step j.
+__device__ __noinline__ void init_chain(const Ctx& cx, const float* __restrict__ st_in, uint32_t j, uint32_t tl, int hf, int dv)
+{
+    cx.wait(B_DECAY_READY0 + (j & 3u), (j >> 2) & 1u);
+    const float wb = cx.misc->decay[j & 3u].wb;
+    tc_fence_after();
+#pragma unroll 1
+    for (int g = 0; g < 4; ++g) {
+        const int c0 = 64 * hf + 16 * g;
+        uint32_t acc[16], pk[8];
+#pragma unroll
+        for (int i = 0; i < 16; ++i) acc[i] = __float_as_uint(st_in[(c0 + i) * 128 + dv]);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) pk[i] = pack_bf16x2(__uint_as_float(acc[2 * i]), __uint_as_float(acc[2 * i + 1]));
+        tmem_st8(tl + TM_SBF + (c0 >> 1), pk);
+#pragma unroll
+        for (int i = 0; i < 16; ++i) acc[i] = __float_as_uint(__uint_as_float(acc[i]) * wb);
+        tmem_st16(tl + TM_S32 + c0, acc);
+    }
+    tmem_st_wait();
+    tc_fence_before();
+}
+
 // ================================================================================================
-// warps 16-23: chain group (Delta epilogue, start states, final states)
+// warps 12-19: chain group (Delta epilogue, state conversion, outputs, final state)
 // ================================================================================================
 __device__ void role_chain(const Ctx& cx, const TcParams& prm, int wtid)
 {
@@ -769,150 +835,112 @@ __device__ void role_chain(const Ctx& cx, const TcParams& prm, int wtid)
     const int dv = w4 * 32 + lane;                        // value-dimension index = TMEM lane
     const uint32_t tl = cx.tmem + ((uint32_t)(w4 * 32) << 16);
     Misc* misc = cx.misc;
-    const bool pair = prm.ng == 2;
+    const uint32_t num_items = (uint32_t)p.num_seqs * (uint32_t)p.Hv;
     const bool has_init = p.init_state != nullptr;
 
-    // items without any chunk (empty requests): the final state is the start state
-    if (p.out_state) {
-        const uint32_t num_items = (uint32_t)p.num_seqs * (uint32_t)(p.Hv / prm.ng);
+    uint32_t j = 0;
 #pragma unroll 1
-        for (int r = 0;; ++r) {
-            const uint32_t item = StepCursor::item_of(r);
-            if (item >= num_items) break;
-            const int4 ci = StepCursor::lookup(&p, prm.s.order, item, prm.ng);
-            if (ci.y > ci.x) continue;
-            for (int m = 0; m < prm.ng; ++m) {
-                const size_t off = ((size_t)ci.w * p.Hv + (ci.z & 0xffff) + m) * 128 * 128;
+    for (int r = 0;; ++r) {
+        const uint32_t item = ChunkCursor::item_of(r);
+        if (item >= num_items) break;
+        const int4 ci = ChunkCursor::lookup(&p, prm.s.order, item);
+        const int n = ci.w, h = ci.z & 0xffff;
+        const int row_begin = ci.x, row_end = ci.y;
+        const int nchunks = (row_end - row_begin + 63) >> 6;
+        const size_t st_off = ((size_t)n * p.Hv + h) * 128 * 128;
+        float* st_out = p.out_state ? p.out_state + st_off : nullptr;
+        if (nchunks == 0) {                                   // empty request: the final state is the start state
+            if (st_out)
                 for (int a = 0; a < 64; ++a)
-                    p.out_state[off + (64 * hf + a) * 128 + dv] = has_init ? p.init_state[off + (64 * hf + a) * 128 + dv] : 0.f;
-            }
+                    st_out[(64 * hf + a) * 128 + dv] = has_init ? p.init_state[st_off + (64 * hf + a) * 128 + dv] : 0.f;
+            continue;
         }
-    }
+        // ---- chain start: the previous chain's final state has been read out (below); a start state, if given, goes
+        // into tensor memory as the first chunk's bf16 operand and, multiplied by the chunk's decay, as the fp32 state
+        if (has_init) init_chain(cx, p.init_state + st_off, j, tl, hf, dv);
+        warp_arrive(cx.bar(B_SBF_READY), lane);               // the start state of step j is in place
+#pragma unroll 1
+        for (int c = 0; c < nchunks; ++c, ++j) {
+            const int row0 = row_begin + c * 64;
+            const int nvalid = min(64, row_end - row0);
+            const bool last = c == nchunks - 1;
+            const Decay& dc = misc->decay[j & 3u];
 
-    // final state of the chain whose last update went into state buffer m: cfin * stored state
-    auto store_final = [&](int n, int h, int m, float cfin) {
-        if (!p.out_state || misc->abort) return;
-        float* st_out = p.out_state + ((size_t)n * p.Hv + h) * 128 * 128;
-        tc_fence_after();
+            // ---- Delta epilogue: bf16 Delta^T and decayed Delta'^T as TMEM A operands ----------------------
+            cx.wait(B_DECAY_READY0 + (j & 3u), (j >> 2) & 1u);   // decay factors of this chunk are published
+            cx.wait(B_MMA1_DONE, j & 1u);
+            tc_fence_after();
 #pragma unroll 1
-        for (int gq = 0; gq < 4; ++gq) {
-            const int c0 = 64 * hf + 16 * gq;
-            uint32_t acc[16];
-            tmem_ld16(tl + TM_S32 + 128u * (uint32_t)m + c0, acc);
-            tmem_ld_wait();
-#pragma unroll
-            for (int e = 0; e < 16; ++e) st_out[(c0 + e) * 128 + dv] = __uint_as_float(acc[e]) * cfin;
-        }
-    };
-    // Start state of a step: the bf16 copy that is the A operand of its MMAs, taken from the chain's stored fp32
-    // state (or from init_state at the chain's first chunk); where the step starts from a rescaled state, the
-    // stored state is multiplied by wb on the way.
-    auto make_start = [&](const StepCursor& sc, uint32_t step) {
-        const bool sfirst = sc.first();
-        if (sfirst && !has_init) return;                     // zero start: the step's MMAs skip the state
-        cx.wait(B_DECAY_READY0 + (step % RD), (step / RD) & 1u);
-        const Decay& dn = misc->decay[step % RD];
-        const float wb = dn.wb;
-        const bool rescale = dn.rescale != 0 || sfirst;
-        const float* st_in = sfirst ? p.init_state + ((size_t)sc.n * p.Hv + sc.h()) * 128 * 128 : nullptr;
-        const uint32_t s32 = tl + TM_S32 + 128u * (uint32_t)sc.m;
-        tc_fence_after();
-#pragma unroll 1
-        for (int gq = 0; gq < 4; ++gq) {
-            const int c0 = 64 * hf + 16 * gq;
-            uint32_t acc[16], pk[8];
-            if (sfirst) {
-#pragma unroll
-                for (int e = 0; e < 16; ++e) acc[e] = __float_as_uint(st_in[(c0 + e) * 128 + dv]);
-            } else {
-                tmem_ld16(s32 + c0, acc);
+            for (int g = 0; g < 2; ++g) {
+                const int c0 = 32 * hf + 16 * g;
+                uint32_t acc[16], d1[8], d2[8];
+                tmem_ld16(tl + TM_ACC1 + c0, acc);
                 tmem_ld_wait();
-            }
 #pragma unroll
-            for (int e = 0; e < 8; ++e) pk[e] = pack_bf16x2(__uint_as_float(acc[2 * e]), __uint_as_float(acc[2 * e + 1]));
-            tmem_st8(tl + TM_SBF + (c0 >> 1), pk);
-            if (rescale) {
-#pragma unroll
-                for (int e = 0; e < 16; ++e) acc[e] = __float_as_uint(__uint_as_float(acc[e]) * wb);
-                tmem_st16(s32 + c0, acc);
+                for (int i4 = 0; i4 < 4; ++i4) {
+                    // the accumulator holds Delta~^T = Delta^T diag(beta)^-1 (see the Gram post-processing): it is the A
+                    // operand of the output product as it stands (P has beta on its columns), and with the factors
+                    // beta e^(G_C - G) / c that of the state update
+                    const float4 er = *reinterpret_cast<const float4*>(&dc.bRest[c0 + 4 * i4]);
+                    const float a0 = __uint_as_float(acc[4 * i4]), a1 = __uint_as_float(acc[4 * i4 + 1]);
+                    const float a2 = __uint_as_float(acc[4 * i4 + 2]), a3 = __uint_as_float(acc[4 * i4 + 3]);
+                    d1[2 * i4] = pack_bf16x2(a0, a1);
+                    d1[2 * i4 + 1] = pack_bf16x2(a2, a3);
+                    d2[2 * i4] = pack_bf16x2(a0 * er.x, a1 * er.y);
+                    d2[2 * i4 + 1] = pack_bf16x2(a2 * er.z, a3 * er.w);
+                }
+                tmem_st8(tl + TM_DBF + c0, d1);
+                tmem_st8(tl + TM_DPBF + c0, d2);
             }
-        }
-        tmem_st_wait();
-        tc_fence_before();
-    };
+            tmem_st_wait();
+            tc_fence_before();
+            const float cfin = dc.cfin;          // read before the arrivals below let the pipeline move on to the slot's reuse
+            warp_arrive(cx.bar(B_D_READY), lane);
 
-    StepCursor cur, nx;
-    cur.init(prm);
-    nx = cur;
-    if (nx.valid) nx.advance();
-    if (cur.valid) {
-        make_start(cur, 0u);
-        warp_arrive(cx.bar(B_SBF_READY), lane);
-    }
-    int pn = 0, ph = 0, pm = 0; float pcfin = 0.f; bool plast = false;       // the step before the current one
-#pragma unroll 1
-    for (uint32_t i = 0; cur.valid; ++i) {
-        const Decay& dc = misc->decay[i % RD];
-        // ---- Delta epilogue: bf16 Delta^T and decayed Delta'^T as TMEM A operands ----------------------
-        cx.wait(B_DECAY_READY0 + (i % RD), (i / RD) & 1u);       // decay factors of this step are published
-        cx.wait(B_MMA1_DONE, i & 1u);
-        tc_fence_after();
-#pragma unroll 1
-        for (int gq = 0; gq < 2; ++gq) {
-            const int c0 = 32 * hf + 16 * gq;
-            uint32_t acc[16], d1[8], d2[8];
-            tmem_ld16(tl + TM_ACC1 + c0, acc);
-            tmem_ld_wait();
-#pragma unroll
-            for (int i4 = 0; i4 < 4; ++i4) {
-                // the accumulator holds Delta~^T = Delta^T diag(beta)^-1 (beta sits on the columns of the solve)
-                const float4 bt = *reinterpret_cast<const float4*>(&dc.beta[c0 + 4 * i4]);
-                const float4 er = *reinterpret_cast<const float4*>(&dc.bRest[c0 + 4 * i4]);
-                const float a0 = __uint_as_float(acc[4 * i4]), a1 = __uint_as_float(acc[4 * i4 + 1]);
-                const float a2 = __uint_as_float(acc[4 * i4 + 2]), a3 = __uint_as_float(acc[4 * i4 + 3]);
-                d1[2 * i4] = pack_bf16x2(a0 * bt.x, a1 * bt.y);
-                d1[2 * i4 + 1] = pack_bf16x2(a2 * bt.z, a3 * bt.w);
-                d2[2 * i4] = pack_bf16x2(a0 * er.x, a1 * er.y);
-                d2[2 * i4 + 1] = pack_bf16x2(a2 * er.z, a3 * er.w);
+            // ---- state: bf16 copy for the next chunk's MMAs, or the final state ------------------------------
+            // if the next chunk starts from a rescaled state, the stored state is multiplied by wb on the way
+            float wb = 1.f;
+            bool rescale = false;
+            if (!last) {
+                cx.wait(B_DECAY_READY0 + ((j + 1) & 3u), ((j + 1) >> 2) & 1u);
+                wb = misc->decay[(j + 1) & 3u].wb;
+                rescale = misc->decay[(j + 1) & 3u].rescale != 0;
             }
-            tmem_st8(tl + TM_DBF + c0, d1);
-            tmem_st8(tl + TM_DPBF + c0, d2);
+            cx.wait(B_STATE_DONE, j & 1u);
+            if (!last) cx.wait(B_SQ_DONE, j & 1u);              // the bf16 state of this chunk has been read for the last time
+            tc_fence_after();
+#pragma unroll 1
+            for (int g = 0; g < 4; ++g) {
+                const int c0 = 64 * hf + 16 * g;
+                uint32_t acc[16];
+                tmem_ld16(tl + TM_S32 + c0, acc);
+                tmem_ld_wait();
+                if (!last) {
+                    uint32_t pk[8];
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) pk[i] = pack_bf16x2(__uint_as_float(acc[2 * i]), __uint_as_float(acc[2 * i + 1]));
+                    tmem_st8(tl + TM_SBF + (c0 >> 1), pk);
+                    if (rescale) {
+#pragma unroll
+                        for (int i = 0; i < 16; ++i) acc[i] = __float_as_uint(__uint_as_float(acc[i]) * wb);
+                        tmem_st16(tl + TM_S32 + c0, acc);
+                    }
+                } else if (st_out && !misc->abort) {
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) st_out[(c0 + i) * 128 + dv] = __uint_as_float(acc[i]) * cfin;
+                }
+            }
+            tmem_st_wait();
+            tc_fence_before();
+            if (!last) warp_arrive(cx.bar(B_SBF_READY), lane);    // (a chain's first chunk is announced at the chain start)
         }
-        tmem_st_wait();
-        tc_fence_before();
-        const float cfin = dc.cfin;          // read before the arrivals below let the ring slot move on
-        // A pair observes the completion of the previous step's state update here: it lies in the past (MMAs
-        // complete in issue order) and must be consumed before this step's update can complete the next phase.
-        if (pair && i >= 1) cx.wait(B_STATE_DONE, (i - 1) & 1u);
-        warp_arrive(cx.bar(B_D_READY), lane);
-        warp_arrive(cx.bar(B_DECAY_FREE0 + (i % RD)), lane);
-        // ---- final states ----------------------------------------------------------------------------------
-        if (pair) {
-            if (plast) store_final(pn, ph, pm, pcfin);
-        } else {
-            cx.wait(B_STATE_DONE, i & 1u);
-            if (cur.last()) store_final(cur.n, cur.h(), cur.m, cfin);
-        }
-        // ---- start state of step i + 1 ----------------------------------------------------------------------
-        if (nx.valid) {
-            cx.wait(B_SQ_DONE, i & 1u);                          // the bf16 state of this step has been read
-            make_start(nx, i + 1);
-            warp_arrive(cx.bar(B_SBF_READY), lane);
-        } else if (pair) {
-            cx.wait(B_STATE_DONE, i & 1u);
-            store_final(cur.n, cur.h(), cur.m, cfin);            // the very last step ends its chain
-        }
-        pn = cur.n; ph = cur.h(); pm = cur.m; pcfin = cfin; plast = cur.last();
-        cur = nx;
-        if (nx.valid) nx.advance();
     }
 }
 
 // ================================================================================================
-// warps 24-27: output group (one warp per TMEM lane window).  Scales S0 Q^T by e^G in place as soon as it is
-// complete, so that Delta^T P^T can accumulate on top, then reads O^T and stores the valid rows off the chain's
-// critical path.  For a fixed token the 128 lanes hold 128 consecutive bf16 of out_o: each warp store writes
-// 64 contiguous bytes (two full sectors), so the outputs go straight from registers to global memory.
+// warps 24-27: output group (one warp per TMEM lane window).  O^T = diag(e^G) (S0 Q^T) + Delta^T P^T of chunk j,
+// read from the two accumulators as soon as the chunk's last MMAs have completed: first everything is read, combined
+// and rounded into registers, which releases the accumulators for the next chunk early; the stores follow.
 // ================================================================================================
 __device__ void role_out(const Ctx& cx, const TcParams& prm, int warp, int lane)
 {
@@ -921,61 +949,65 @@ __device__ void role_out(const Ctx& cx, const TcParams& prm, int warp, int lane)
     const int dv = w4 * 32 + lane;
     const uint32_t tl = cx.tmem + ((uint32_t)(w4 * 32) << 16);
     __nv_bfloat16* __restrict__ og = reinterpret_cast<__nv_bfloat16*>(p.out_o);
-    const bool has_init = p.init_state != nullptr;
-    StepCursor cc;
-    cc.init(prm);
+    ChunkCursor cc;
+    cc.init(&p, prm.s.order);
 #pragma unroll 1
-    for (uint32_t i = 0; cc.valid; ++i, cc.advance()) {
+    for (uint32_t j = 0; cc.valid; ++j, cc.advance()) {
         const int row0 = cc.row0(), nvalid = cc.nvalid();
-        const bool has_state = !cc.first() || has_init;
-        const Decay& dc = cx.misc->decay[i % RD];
-        cx.wait(B_DECAY_READY0 + (i % RD), (i / RD) & 1u);
-        if (has_state) {
-            cx.wait(B_SQ_DONE, i & 1u);
-            tc_fence_after();
-#pragma unroll 1
-            for (int gq = 0; gq < 4; ++gq) {
-                const int c0 = 16 * gq;
-                uint32_t a2[16];
-                tmem_ld16(tl + TM_ACC2 + c0, a2);
-                tmem_ld_wait();
-#pragma unroll
-                for (int i4 = 0; i4 < 4; ++i4) {
-                    const float4 eg = *reinterpret_cast<const float4*>(&dc.eG[c0 + 4 * i4]);
-                    a2[4 * i4 + 0] = __float_as_uint(__uint_as_float(a2[4 * i4 + 0]) * eg.x);
-                    a2[4 * i4 + 1] = __float_as_uint(__uint_as_float(a2[4 * i4 + 1]) * eg.y);
-                    a2[4 * i4 + 2] = __float_as_uint(__uint_as_float(a2[4 * i4 + 2]) * eg.z);
-                    a2[4 * i4 + 3] = __float_as_uint(__uint_as_float(a2[4 * i4 + 3]) * eg.w);
-                }
-                tmem_st16(tl + TM_ACC2 + c0, a2);
-            }
-            tmem_st_wait();
-            tc_fence_before();
-        }
-        warp_arrive(cx.bar(B_ACC2_SCALED), lane);
-        warp_arrive(cx.bar(B_DECAY_FREE0 + (i % RD)), lane);    // last read of this step's decay factors
-        cx.wait(B_MMA3_DONE, i & 1u);
+        const bool first = cc.first() && p.init_state == nullptr;      // zero start state: S0 Q^T was not computed
+        const Decay& dc = cx.misc->decay[j & 3u];
+        cx.wait(B_DECAY_READY0 + (j & 3u), (j >> 2) & 1u);
+        cx.wait(B_MMA3_DONE, j & 1u);
         tc_fence_after();
-        const bool store = og != nullptr && !cx.misc->abort;
-        __nv_bfloat16* optr = og + ((size_t)row0 * p.Hv + cc.h()) * 128 + dv;
+        // For a fixed token the 128 lanes hold 128 consecutive bf16 of out_o: each warp store writes 64 contiguous bytes
+        // (two full sectors), so the outputs go straight from registers to global memory, 16 tokens at a time.
+        uint16_t* optr = reinterpret_cast<uint16_t*>(og) + ((size_t)row0 * p.Hv + cc.h) * 128 + dv;
         const uint32_t ostride = (uint32_t)p.Hv * 128u;
+        const bool full = nvalid == 64;
 #pragma unroll 1
-        for (int gq = 0; gq < 4; ++gq) {
-            const int c0 = 16 * gq;
-            uint32_t a3[16];
-            tmem_ld16(tl + TM_ACC2 + c0, a3);
+        for (int g = 0; g < 4; ++g) {
+            const int c0 = 16 * g;
+            uint32_t a3[16], a2[16];
+            tmem_ld16(tl + TM_ACC3 + c0, a3);
+            if (!first) tmem_ld16(tl + TM_ACC2 + c0, a2);
             tmem_ld_wait();
-            if (gq == 3) {
-                // the accumulator has been read: the chain may overwrite it while the last block is stored
+            if (g == 3) {
+                // both accumulators have been read: the chain may overwrite them while the last block is stored
                 tc_fence_before();
-                warp_arrive(cx.bar(B_ACC2_FREE), lane);
+                warp_arrive(cx.bar(B_ACC23_FREE), lane);
             }
-            if (store) {
+            uint32_t pk[8];
 #pragma unroll
-                for (int e = 0; e < 16; ++e)
-                    if (c0 + e < nvalid) optr[(uint32_t)(c0 + e) * ostride] = __float2bfloat16_rn(__uint_as_float(a3[e]));
+            for (int i4 = 0; i4 < 4; ++i4) {
+                const float4 eg = *reinterpret_cast<const float4*>(&dc.eG[c0 + 4 * i4]);
+                float o0 = __uint_as_float(a3[4 * i4]), o1 = __uint_as_float(a3[4 * i4 + 1]);
+                float o2 = __uint_as_float(a3[4 * i4 + 2]), o3 = __uint_as_float(a3[4 * i4 + 3]);
+                if (!first) {
+                    o0 = fmaf(eg.x, __uint_as_float(a2[4 * i4]), o0); o1 = fmaf(eg.y, __uint_as_float(a2[4 * i4 + 1]), o1);
+                    o2 = fmaf(eg.z, __uint_as_float(a2[4 * i4 + 2]), o2); o3 = fmaf(eg.w, __uint_as_float(a2[4 * i4 + 3]), o3);
+                }
+                pk[2 * i4] = pack_bf16x2(o0, o1);
+                pk[2 * i4 + 1] = pack_bf16x2(o2, o3);
             }
+            if (og) {
+                // a full chunk (all but a request's last) stores without per-token predicates
+                if (full) {
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) {
+                        optr[(uint32_t)(2 * i) * ostride] = (uint16_t)(pk[i] & 0xffffu);
+                        optr[(uint32_t)(2 * i + 1) * ostride] = (uint16_t)(pk[i] >> 16);
+                    }
+                } else {
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) {
+                        if (c0 + 2 * i < nvalid) optr[(uint32_t)(2 * i) * ostride] = (uint16_t)(pk[i] & 0xffffu);
+                        if (c0 + 2 * i + 1 < nvalid) optr[(uint32_t)(2 * i + 1) * ostride] = (uint16_t)(pk[i] >> 16);
+                    }
+                }
+            }
+            optr += 16u * ostride;
         }
+        warp_arrive(cx.bar(B_DECAY_FREE0 + (j & 3u)), lane);    // last read of this chunk's decay factors
     }
 }
 
@@ -997,45 +1029,42 @@ gdn_tc_kernel(const TcParams prm, const __grid_constant__ CUtensorMap tm_q,
     }
     if (tid == 32) {
         for (int i = 0; i < NUM_BARS; ++i) {
-            // arrivals per phase: one per warp of the arriving group, or one tcgen05.commit / TMA transaction
-            uint32_t cnt = 1u;
-            if (i == B_GRAM_FREE) cnt = 4u * (uint32_t)prm.ng;                     // the teams of the tile's steps
-            else if (i >= B_DECAY_FREE0 && i < B_DECAY_FREE0 + (int)RD) cnt = 12u;  // chain and output groups
-            else if ((i >= B_TP_READY0 && i < B_TP_READY0 + (int)RTP) || (i >= B_PRE_DONE0 && i < B_PRE_DONE0 + 3)) cnt = 4u;   // a team
-            else if (i == B_D_READY || i == B_SBF_READY) cnt = 8u;                 // chain group
-            else if (i == B_ACC2_SCALED || i == B_ACC2_FREE) cnt = 4u;             // output group
-            mbar_init(cx.bar(i), cnt);
+            // arrivals per phase: one per warp of the arriving group (G1 and chain: 8 warps, G2: 2 warps)
+            const bool wg_bar = i == B_GRAM_READ || i == B_D_READY || i == B_SBF_READY ||
+                                i == B_WACC_READ || i == B_PRE_DONE0 || i == B_PRE_DONE1 ||
+                                i == B_A_READY0 || i == B_A_READY1 || i == B_A_READY2;
+            const bool out_bar = i == B_ACC23_FREE || (i >= B_DECAY_FREE0 && i <= B_DECAY_FREE3);
+            const bool g2_bar = i == B_TP_READY0 || i == B_TP_READY1 || i == B_TP_READY2;
+            mbar_init(cx.bar(i), wg_bar ? 8u : out_bar ? 4u : g2_bar ? 2u : 1u);
         }
         fence_mbar_init();
         cx.misc->abort = 0u;
         cx.misc->timeout_ns = prm.wait_timeout_ns;
         prefetch_tmap(&tm_q); prefetch_tmap(&tm_k); prefetch_tmap(&tm_v);
     }
-    // the operand tiles P^ and P (contiguous rings) are only ever written on and below their diagonal 16 x 16
+    // the operand tiles T' (3), T'' and P (3), contiguous, are only ever written on and below their 16 x 16 diagonal
     // blocks: everything else is zeroed once, here
-    for (uint32_t i = tid; i < (RTP + RP) * 8192u / 16u; i += kThreads)
+    for (uint32_t i = tid; i < 7u * 8192u / 16u; i += kThreads)
         *reinterpret_cast<uint4*>(cx.sm + SM_TP + i * 16u) = make_uint4(0u, 0u, 0u, 0u);
-    if (tid < 64) cx.misc->ones[tid] = 1.f;
     fence_proxy_async_smem();
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     cx.tmem = cx.misc->tmem_base;
 
-    if (warp == 0) {
-        role_producer(cx, prm, &tm_q, &tm_k, &tm_v);
-    } else if (warp == 1) {
-        role_mma_chain(cx, prm);
-    } else if (warp == 2) {
-        role_mma_gram(cx, prm);
-    } else if (warp == 3) {
-        role_decay(cx, prm);
-    } else if (warp < 16) {
-        role_team(cx, prm, (warp - 4) >> 2, warp & 3, lane);
-    } else if (warp < 24) {
-        role_chain(cx, prm, tid - 512);
-    } else {
+    if (warp < 4) {
+        if (warp == 0) role_producer(cx, prm, &tm_q, &tm_k, &tm_v);
+        else if (warp == 1) role_mma_chain(cx, prm);
+        else if (warp == 2) role_mma_gram(cx, prm);
+        else role_decay(cx, prm);
+    } else if (warp >= 24) {
         role_out(cx, prm, warp, lane);
+    } else if (warp < 12) {
+        role_g1(cx, prm, tid - 128);
+    } else if (warp < 20) {
+        role_chain(cx, prm, tid - 384);
+    } else {
+        role_g2(cx, prm, (tid - 640) & 63, (warp - 20) >> 1);
     }
 
     tc_fence_before();
@@ -1086,6 +1115,7 @@ int32_t g_skip_kq_load = -1;
 
 }  // namespace
 
+
 extern "C" GDN_API void gdn_test_hooks(uint64_t wait_timeout_ns, int32_t skip_kq_load_of_chunk)
 {
     g_wait_timeout_ns = wait_timeout_ns ? wait_timeout_ns : 2000000000ull;
@@ -1097,7 +1127,7 @@ bool tcgen05_supported(const Problem& p)
     return p.dk == 128 && p.dv == 128 && p.total_tokens > 0;
 }
 
-cudaError_t launch_tcgen05(const Problem& p, const Sched& s, int pairing, cudaStream_t stream, int* launches)
+cudaError_t launch_tcgen05(const Problem& p, const Sched& s, cudaStream_t stream, int* launches)
 {
     if (!tcgen05_supported(p)) return cudaErrorNotSupported;
     CUtensorMap tq, tk, tv;
@@ -1116,15 +1146,10 @@ cudaError_t launch_tcgen05(const Problem& p, const Sched& s, int pairing, cudaSt
     }
     e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     if (e != cudaSuccess) return e;
-    // Pairs need an even number of v-heads per q/k head.  With no more chains than SMs every chain gets an SM of
-    // its own, which is faster than sharing one; beyond that, two sibling chains per CTA overlap each other.
-    const bool can_pair = ((p.Hv / p.Hq) % 2) == 0;
-    const long long chains = (long long)p.num_seqs * p.Hv;
-    const bool pair = can_pair && (pairing == 2 || (pairing == 0 && chains > sms));
-    long long grid = pair ? chains / 2 : chains;
+    long long grid = (long long)p.num_seqs * p.Hv;
     if (grid > sms) grid = sms;
     TcParams prm;
-    prm.p = p; prm.s = s; prm.ng = pair ? 2 : 1;
+    prm.p = p; prm.s = s;
     prm.wait_timeout_ns = g_wait_timeout_ns; prm.skip_kq_load = g_skip_kq_load;
     g_skip_kq_load = -1;                                        // one-shot: consumed by this launch
     gdn_tc_kernel<<<(unsigned)grid, kThreads, SMEM_BYTES, stream>>>(prm, tq, tk, tv);

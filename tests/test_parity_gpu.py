@@ -13,7 +13,6 @@ from gpu_utils import run_library, assert_parity, assert_parity_lean, state_rel_
 pytestmark = pytest.mark.gpu
 
 SIMT, TC = 1, 2
-TC_SINGLE, TC_PAIR = 3, 4          # the tensor-core path with its work split fixed: one chain / a sibling pair per CTA
 
 
 def check(inp, kernel, **kw):
@@ -55,28 +54,26 @@ def test_simt_init_state_resume():
     assert np.abs(o_tail - ro[120:]).max() < 1e-4
 
 
-@pytest.mark.parametrize("kernel", [SIMT, TC, TC_SINGLE, TC_PAIR, 0])
+@pytest.mark.parametrize("kernel", [SIMT, TC, 0])
 def test_bf16_d128_ragged_batch(kernel):
     lens = [130, 64, 1, 0, 63, 65, 127, 128, 129, 410, 5]
     inp = make_inputs(lens, 2, 4, 128, 128, "bf16", seed=77)
     check(inp, kernel)
 
 
-@pytest.mark.parametrize("kernel", [SIMT, TC, TC_PAIR])
+@pytest.mark.parametrize("kernel", [SIMT, TC])
 def test_config1_single_layer(kernel):
     check(config_single_layer(), kernel)
 
 
-@pytest.mark.parametrize("kernel", [TC, TC_SINGLE, TC_PAIR])
+@pytest.mark.parametrize("kernel", [TC])
 def test_gqa_group_sizes(kernel):
     for Hq, Hv in [(1, 1), (1, 4), (3, 3), (2, 6), (2, 8)]:
-        if kernel == TC_PAIR and (Hv // Hq) % 2:
-            continue                                       # pairs need an even number of v-heads per q/k head
         inp = make_inputs([200, 77], Hq, Hv, 128, 128, "bf16", seed=5 + Hq * 10 + Hv)
         check(inp, kernel)
 
 
-@pytest.mark.parametrize("kernel", [TC_SINGLE, TC_PAIR])
+@pytest.mark.parametrize("kernel", [TC])
 def test_tc_init_state_resume_ragged(kernel):
     """Resume identity on the tensor-core path: run(prefix + tail) == run(tail, init = run(prefix)), request by
     request on a ragged batch that includes empty tails (whose final state must equal the start state) and
@@ -108,7 +105,7 @@ def test_tc_init_state_resume_ragged(kernel):
             np.testing.assert_array_equal(st_res[n], st_pre[n].astype(np.float32).astype(np.float64))
 
 
-@pytest.mark.parametrize("kernel", [SIMT, TC_SINGLE, TC_PAIR])
+@pytest.mark.parametrize("kernel", [SIMT, TC])
 def test_run_to_run_bitwise_determinism(kernel):
     inp = make_inputs([100, 37, 200], 2, 4, 128, 128, "bf16", seed=9)
     o1, s1, _ = run_library(inp, kernel=kernel)
@@ -117,7 +114,7 @@ def test_run_to_run_bitwise_determinism(kernel):
     np.testing.assert_array_equal(s1, s2)
 
 
-@pytest.mark.parametrize("kernel", [SIMT, TC_SINGLE, TC_PAIR])
+@pytest.mark.parametrize("kernel", [SIMT, TC])
 def test_guard_rows_around_outputs_stay_untouched(kernel):
     """out_o sits between 64 guard rows on each side and out_state between two guard states, all filled with a
     bit pattern; ragged last chunks (whose 64-row tiles reach past the request and past the end of the batch)
@@ -151,7 +148,7 @@ def _poison_other_requests(inp, keep):
     return p
 
 
-@pytest.mark.parametrize("kernel", [SIMT, TC_SINGLE, TC_PAIR])
+@pytest.mark.parametrize("kernel", [SIMT, TC])
 def test_poisoned_neighbour_rows_do_not_leak(kernel):
     """The 64-row tiles of a request's ragged last chunk overlap the first rows of the next request (and a
     short request sits inside tiles of its neighbours).  Filling every foreign row with large finite values
@@ -185,7 +182,7 @@ def test_host_memory_call(kernel):
     assert_parity(inp, o, st, ro, rst)
 
 
-@pytest.mark.parametrize("kernel", [SIMT, TC_SINGLE, TC_PAIR])
+@pytest.mark.parametrize("kernel", [SIMT, TC])
 def test_strong_decay_and_beta_zero(kernel):
     """alpha -> 0 keeps only the last token's rank-1 update; beta = 0 keeps the state at zero."""
     inp = make_inputs([130], 1, 2, 128, 128, "bf16", seed=41)
@@ -206,13 +203,13 @@ def test_strong_decay_and_beta_zero(kernel):
     assert_parity(inp, o, st, ro, rst)
 
 
-@pytest.mark.parametrize("kernel", [SIMT, TC_SINGLE, TC_PAIR])
+@pytest.mark.parametrize("kernel", [SIMT, TC])
 def test_weak_decay_long_memory(kernel):
     inp = make_inputs([700], 1, 2, 128, 128, "bf16", seed=43, g_lo=-0.002, g_hi=-0.0001)
     check(inp, kernel)
 
 
-@pytest.mark.parametrize("kernel", [TC, TC_SINGLE])
+@pytest.mark.parametrize("kernel", [TC])
 def test_config3_concurrent_hits_full_size_all_chains(kernel):
     """Full-size 32-request batch in the benchmark's launch configuration: every one of the 1,024 chains
     (all outputs, all final states) against the oracle."""
@@ -291,7 +288,7 @@ def test_weak_decay_tail_vs_full_bound_has_teeth(kernel):
         assert bound > 0.1                                   # the bound is not vacuous here
 
 
-@pytest.mark.parametrize("kernel", [TC_SINGLE, TC_PAIR])
+@pytest.mark.parametrize("kernel", [TC])
 def test_randomised_ragged_batches(kernel):
     """Seeded sweep over ragged batches: request counts 1-11, lengths 0-330 (plus runs of lengths around one chunk and
     one long request), seven head configurations, four decay ranges from very weak to very strong.  The pipeline of
@@ -309,8 +306,6 @@ def test_randomised_ragged_batches(kernel):
         if sum(lens) == 0:
             lens[0] = 5
         hq, g = heads[it % 7]
-        if kernel == TC_PAIR and g % 2:
-            g += 1                                         # pairs need an even number of v-heads per q/k head
         g_lo, g_hi = decay[it % 4]
         inp = make_inputs(lens, hq, hq * g, 128, 128, "bf16", seed=2608030310 + 50_000 + it, g_lo=g_lo, g_hi=g_hi)
         check(inp, kernel)
