@@ -30,7 +30,7 @@
  * init_state) is a host pointer (pinned memory makes the copies asynchronous); the library
  * stages through the caller's workspace and copies results back on the same stream.
  * Ownership: every buffer is the caller's.  The library allocates no device memory, keeps no
- * state between calls and frees nothing.  Calls are asynchronous on desc->stream; buffers
+ * state between calls and frees nothing (the one exception, gdn_tail_replay_static_scratch, says so below).  Calls are asynchronous on desc->stream; buffers
  * must stay alive until the stream has passed the call.  Valid output rows are fully
  * overwritten; no other byte of the outputs is touched.  A request of length 0 gets a zero
  * state (or its init_state) and no output rows.
@@ -120,6 +120,22 @@ GDN_API int32_t gdn_tail_replay(const gdn_desc* desc, const void* q, const void*
 GDN_API int32_t gdn_full_prefill(const gdn_desc* desc, const void* q, const void* k, const void* v,
                          const float* g, const float* beta, const int32_t* cu_tail_lens,
                          int32_t chunk, void* out_o, float* out_state);
+
+/*
+ * One decoding step from a given state (paper, Method section: after the replay "the model continues serving the
+ * current request ... with the retrieved FA KV and reconstructed linear-attention states", i.e. Eq. 1 continued
+ * one token at a time from the rebuilt state).  Every request contributes exactly one token:
+ *     q, k [N, Hq, dk], v [N, Hv, dv] in io_dtype; g, beta [N, Hv] fp32;
+ *     state_in, state_out [N, Hv, dk, dv] fp32 in the layout of out_state (they may be the same buffer);
+ *     out_o [N, Hv, dv] in io_dtype, or NULL.
+ * desc supplies the head counts and dims (dk, dv in {64, 128}), io_dtype, num_seqs = N and the stream;
+ * total_tokens, workspace, init_state and kernel are ignored.  Device pointers only (GDN_MEM_HOST: UNSUPPORTED).
+ * It is gdn_tail_replay with init_state = state_in and one-row requests, as a kernel of its own because it is bound
+ * by reading and writing the states once, not by the chunk machinery.
+ */
+GDN_API int32_t gdn_decode_step(const gdn_desc* desc, const void* q, const void* k, const void* v,
+                                const float* g, const float* beta, const float* state_in,
+                                void* out_o, float* state_out);
 
 /*
  * Tail replay for callers that have no device memory to hand over as workspace.  (The paper has no

@@ -8,11 +8,12 @@ from ._binding import (  # noqa: F401
     GdnDesc, GDN_OK, GDN_F32, GDN_BF16, GDN_MEM_DEVICE, GDN_MEM_HOST,
     GDN_KERNEL_AUTO, GDN_KERNEL_FP32_SIMT, GDN_KERNEL_TCGEN05,
     GdnError, library_path, load_library, status_string, tail_select, workspace_size,
-    gdn_tail_replay, gdn_full_prefill, gdn_tail_replay_static_scratch, last_launch_count, Workspace, test_hooks,
+    gdn_tail_replay, gdn_full_prefill, gdn_tail_replay_static_scratch, gdn_decode_step, last_launch_count, Workspace,
+    test_hooks,
 )
 
 __all__ = [
     "GdnDesc", "GdnError", "library_path", "load_library", "status_string", "tail_select",
-    "workspace_size", "gdn_tail_replay", "gdn_full_prefill", "gdn_tail_replay_static_scratch",
+    "workspace_size", "gdn_tail_replay", "gdn_full_prefill", "gdn_tail_replay_static_scratch", "gdn_decode_step",
     "last_launch_count", "Workspace",
 ]

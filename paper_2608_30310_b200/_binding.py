@@ -57,6 +57,8 @@ def load_library():
         fn = getattr(lib, name)
         fn.restype = ctypes.c_int32
         fn.argtypes = fwd_args
+    lib.gdn_decode_step.restype = ctypes.c_int32
+    lib.gdn_decode_step.argtypes = [dp, vp, vp, vp, vp, vp, vp, vp, vp]
     lib.tail_select.restype = ctypes.c_int64
     lib.tail_select.argtypes = [ctypes.c_int64, ctypes.c_double]
     lib.gdn_status_string.restype = ctypes.c_char_p
@@ -188,3 +190,39 @@ def gdn_tail_replay_static_scratch(q, k, v, g, beta, cu_tail_lens, chunk, out_o,
 def gdn_full_prefill(q, k, v, g, beta, cu_tail_lens, chunk, out_o, out_state, **kw) -> int:
     """Full prefill (paper Eq. 1 over whole prefixes); same arguments as ``gdn_tail_replay``."""
     return _forward("gdn_full_prefill", q, k, v, g, beta, cu_tail_lens, chunk, out_o, out_state, **kw)
+
+
+def gdn_decode_step(q, k, v, g, beta, state_in, out_o, state_out, *, stream=None, check: bool = True) -> int:
+    """One token per request from a given state (Eq. 1 continued after the replay); see the header.
+
+    q, k [N, Hq, dk], v [N, Hv, dv], g, beta [N, Hv], state_in / state_out [N, Hv, dk, dv] fp32 (may be the
+    same tensor), out_o [N, Hv, dv] or None.  Device tensors only."""
+    import torch
+    lib = load_library()
+    N, Hq, dk = q.shape
+    _, Hv, dv = v.shape
+    if q.dtype == torch.bfloat16:
+        io = GDN_BF16
+    elif q.dtype == torch.float32:
+        io = GDN_F32
+    else:
+        raise TypeError("q, k, v must be bfloat16 or float32")
+    for name, t, shape, dt in (("k", k, (N, Hq, dk), q.dtype), ("v", v, (N, Hv, dv), q.dtype), ("g", g, (N, Hv), torch.float32),
+                               ("beta", beta, (N, Hv), torch.float32), ("state_in", state_in, (N, Hv, dk, dv), torch.float32),
+                               ("state_out", state_out, (N, Hv, dk, dv), torch.float32)):
+        if tuple(t.shape) != shape or t.dtype != dt or not t.is_contiguous() or not t.is_cuda:
+            raise ValueError("%s must be a contiguous device tensor of shape %s and dtype %s" % (name, shape, dt))
+    if out_o is not None and (tuple(out_o.shape) != (N, Hv, dv) or out_o.dtype != q.dtype or not out_o.is_cuda):
+        raise ValueError("out_o must be [N, Hv, dv] in the io dtype on the device")
+    desc = GdnDesc()
+    desc.num_qk_heads, desc.num_v_heads, desc.head_k_dim, desc.head_v_dim = Hq, Hv, dk, dv
+    desc.io_dtype, desc.num_seqs, desc.total_tokens = io, N, N
+    desc.memory, desc.kernel = GDN_MEM_DEVICE, GDN_KERNEL_AUTO
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    desc.stream = int(stream.cuda_stream)
+    rc = int(lib.gdn_decode_step(ctypes.byref(desc), _ptr(q), _ptr(k), _ptr(v), _ptr(g), _ptr(beta), _ptr(state_in),
+                                 _ptr(out_o), _ptr(state_out)))
+    if check and rc != GDN_OK:
+        raise GdnError(rc, "gdn_decode_step")
+    return rc

@@ -9,7 +9,7 @@ PKG = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "libgdn_tail_replay.so")
-SOURCES = ["api.cu", "sched.cu", "gdn_simt.cu", "gdn_tc.cu"]
+SOURCES = ["api.cu", "sched.cu", "gdn_simt.cu", "gdn_tc.cu", "gdn_decode.cu"]
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
     "--expt-relaxed-constexpr", "-Xcompiler", "-fPIC", "-Xcompiler", "-fvisibility=hidden",

@@ -213,6 +213,28 @@ int32_t gdn_tail_replay_static_scratch(const gdn_desc* desc, const void* q, cons
     return forward(&d, q, k, v, g, beta, cu_tail_lens, chunk, out_o, out_state);
 }
 
+int32_t gdn_decode_step(const gdn_desc* d, const void* q, const void* k, const void* v, const float* g,
+                        const float* beta, const float* state_in, void* out_o, float* state_out)
+{
+    g_last_launches = 0;
+    if (!desc_shape_ok(d)) return GDN_ERR_INVALID_ARG;
+    if (!q || !k || !v || !g || !beta || !state_in || !state_out) return GDN_ERR_INVALID_ARG;
+    if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(g) || !aligned16(beta) ||
+        !aligned16(state_in) || !aligned16(state_out) || !aligned16(out_o))
+        return GDN_ERR_INVALID_ARG;
+    const bool dims_ok = (d->head_k_dim == 64 || d->head_k_dim == 128) && (d->head_v_dim == 64 || d->head_v_dim == 128);
+    if (!dims_ok) return GDN_ERR_UNSUPPORTED;
+    if (d->memory != GDN_MEM_DEVICE) return GDN_ERR_UNSUPPORTED;
+    if (d->num_seqs == 0) return GDN_OK;
+    const cudaError_t e = gdn::launch_decode(q, k, v, g, beta, state_in, state_out, out_o, d->num_seqs, d->num_qk_heads,
+                                             d->num_v_heads, d->head_k_dim, d->head_v_dim, d->io_dtype,
+                                             (cudaStream_t)d->stream);
+    if (e == cudaErrorNotSupported) return GDN_ERR_UNSUPPORTED;
+    if (e != cudaSuccess) return GDN_ERR_CUDA;
+    g_last_launches = 1;
+    return GDN_OK;
+}
+
 int64_t tail_select(int64_t prefix_len, double budget_frac)
 {
     if (prefix_len < 0 || budget_frac != budget_frac || budget_frac < 0.0) return -1;

@@ -43,5 +43,9 @@ cudaError_t launch_simt(const Problem& p, const Sched& s, int io_dtype, cudaStre
 // Whether the tensor-core path can run this problem; launch_tcgen05 returns cudaErrorNotSupported when it cannot.
 bool tcgen05_supported(const Problem& p);
 cudaError_t launch_tcgen05(const Problem& p, const Sched& s, cudaStream_t stream, int* launches);
+// One token per request from a given state (state_in and state_out may alias).
+cudaError_t launch_decode(const void* q, const void* k, const void* v, const float* g, const float* beta,
+                          const float* state_in, float* state_out, void* out_o, int32_t num_seqs, int32_t Hq,
+                          int32_t Hv, int32_t dk, int32_t dv, int io_dtype, cudaStream_t stream);
 
 }  // namespace gdn
