@@ -28,7 +28,11 @@
  * Memory.  With desc->memory == GDN_MEM_DEVICE every data pointer is a device pointer.  With
  * GDN_MEM_HOST every data pointer (q, k, v, g, beta, cu_tail_lens, out_o, out_state,
  * init_state) is a host pointer (pinned memory makes the copies asynchronous); the library
- * stages through the caller's workspace and copies results back on the same stream.
+ * stages through the caller's workspace, pipelined by groups of requests: inputs travel host to
+ * device on one internal copy stream and results device to host on another while the kernels
+ * run on desc->stream, which is also where the call ends (work enqueued on desc->stream after
+ * the call sees the results).  The two copy streams and a few events are created once per
+ * device on the first host-memory call; they are host-side objects, not device memory.
  * Ownership: every buffer is the caller's.  The library allocates no device memory, keeps no
  * state between calls and frees nothing (the one exception, gdn_tail_replay_static_scratch, says so below).  Calls are asynchronous on desc->stream; buffers
  * must stay alive until the stream has passed the call.  Valid output rows are fully

@@ -57,6 +57,58 @@ size_t sched_bytes(const gdn_desc* d)
     return sizeof(gdn::SchedHeader) + round256((size_t)(d->num_seqs > 0 ? d->num_seqs : 1) * sizeof(int32_t));
 }
 
+// Scheduler + forward kernel of one (sub-)batch on `stream`; sets the launch count of this thread.
+int32_t run_kernels(gdn::Problem& p, gdn::Sched sched, bool use_tc, int32_t kernel, int32_t io_dtype, cudaStream_t stream)
+{
+    g_last_launches = 0;
+    // A single request needs no ordering: the tensor-core path then runs without the scheduler kernel, which
+    // matters for the batch-1 state rebuild (one call per layer, a few microseconds each).
+    if (use_tc && p.num_seqs == 1 && gdn::tcgen05_supported(p)) {
+        sched.order = nullptr;
+    } else {
+        if (gdn::launch_scheduler(p.cu, p.num_seqs, sched, stream) != cudaSuccess) return GDN_ERR_CUDA;
+        g_last_launches += 1;
+    }
+    cudaError_t e = cudaErrorNotSupported;
+    if (use_tc) {
+        e = gdn::launch_tcgen05(p, sched, stream, &g_last_launches);
+        if (e == cudaErrorNotSupported && kernel == GDN_KERNEL_TCGEN05) return GDN_ERR_UNSUPPORTED;
+    }
+    if (e == cudaErrorNotSupported) e = gdn::launch_simt(p, sched, io_dtype, stream, &g_last_launches);
+    if (e == cudaErrorNotSupported) return GDN_ERR_UNSUPPORTED;
+    return e == cudaSuccess ? GDN_OK : GDN_ERR_CUDA;
+}
+
+// Copy streams and events of the host-memory mode, made once per device on its first host-memory call (host-side
+// objects only: no device memory is allocated).
+constexpr int kMaxGroups = 16;
+struct HostPipe {
+    cudaStream_t s_in, s_out;
+    cudaEvent_t ev_start, ev_done, ev_in[kMaxGroups], ev_k[kMaxGroups];
+};
+HostPipe* host_pipe()
+{
+    static HostPipe pipes[kMaxDevices];
+    static bool ready[kMaxDevices] = {};
+    static std::mutex mu;
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return nullptr;
+    std::lock_guard<std::mutex> lock(mu);
+    if (!ready[dev]) {
+        HostPipe& hp = pipes[dev];
+        bool ok = cudaStreamCreateWithFlags(&hp.s_in, cudaStreamNonBlocking) == cudaSuccess &&
+                  cudaStreamCreateWithFlags(&hp.s_out, cudaStreamNonBlocking) == cudaSuccess &&
+                  cudaEventCreateWithFlags(&hp.ev_start, cudaEventDisableTiming) == cudaSuccess &&
+                  cudaEventCreateWithFlags(&hp.ev_done, cudaEventDisableTiming) == cudaSuccess;
+        for (int i = 0; ok && i < kMaxGroups; ++i)
+            ok = cudaEventCreateWithFlags(&hp.ev_in[i], cudaEventDisableTiming) == cudaSuccess &&
+                 cudaEventCreateWithFlags(&hp.ev_k[i], cudaEventDisableTiming) == cudaSuccess;
+        if (!ok) return nullptr;
+        ready[dev] = true;
+    }
+    return &pipes[dev];
+}
+
 int32_t forward(const gdn_desc* d, const void* q, const void* k, const void* v, const float* g,
                 const float* beta, const int32_t* cu, int32_t chunk, void* out_o, float* out_state)
 {
@@ -98,59 +150,92 @@ int32_t forward(const gdn_desc* d, const void* q, const void* k, const void* v, 
     p.num_seqs = d->num_seqs; p.Hq = d->num_qk_heads; p.Hv = d->num_v_heads;
     p.dk = d->head_k_dim; p.dv = d->head_v_dim; p.total_tokens = d->total_tokens;
     p.status_word = d->status_word;
+    const bool use_tc = tc_shape && d->kernel != GDN_KERNEL_FP32_SIMT;
 
-    const Sizes sz = sizes_of(d);
-    void* o_stage = nullptr; float* st_stage = nullptr;
-    if (d->memory == GDN_MEM_HOST) {
-        auto stage_in = [&](const void* src, size_t bytes, cudaError_t& err) -> void* {
-            void* dst = ws;
-            ws += round256(bytes);
-            if (err == cudaSuccess && bytes) err = cudaMemcpyAsync(dst, src, bytes, cudaMemcpyHostToDevice, stream);
-            return dst;
-        };
-        cudaError_t err = cudaSuccess;
-        p.cu = (const int32_t*)stage_in(cu, sz.cu, err);
-        p.q = stage_in(q, sz.qk, err);
-        p.k = stage_in(k, sz.qk, err);
-        p.v = stage_in(v, sz.v, err);
-        p.g = (const float*)stage_in(g, sz.gb, err);
-        p.beta = (const float*)stage_in(beta, sz.gb, err);
-        if (d->init_state) p.init_state = (const float*)stage_in(d->init_state, sz.state, err);
-        if (out_o) { o_stage = ws; ws += round256(sz.o); }
-        if (out_state) { st_stage = (float*)ws; ws += round256(sz.state); }
-        p.out_o = o_stage; p.out_state = st_stage;
-        if (err != cudaSuccess) return GDN_ERR_CUDA;
-    } else {
+    if (d->memory == GDN_MEM_DEVICE) {
         p.q = q; p.k = k; p.v = v; p.g = g; p.beta = beta; p.cu = cu;
         p.init_state = d->init_state; p.out_o = out_o; p.out_state = out_state;
+        return run_kernels(p, sched, use_tc, d->kernel, d->io_dtype, stream);
     }
 
-    const bool use_tc = tc_shape && d->kernel != GDN_KERNEL_FP32_SIMT;
-    // A single request needs no ordering: the tensor-core path then runs without the scheduler kernel, which
-    // matters for the batch-1 state rebuild (one call per layer, a few microseconds each).
-    if (use_tc && p.num_seqs == 1 && gdn::tcgen05_supported(p)) {
-        sched.order = nullptr;
-    } else {
-        if (gdn::launch_scheduler(p.cu, p.num_seqs, sched, stream) != cudaSuccess) return GDN_ERR_CUDA;
-        g_last_launches += 1;
-    }
+    // ---- host memory: staged through the workspace and pipelined by groups of requests over three streams: the
+    // inputs of group i + 1 go host -> device on a copy stream while group i computes on the caller's stream and the
+    // results of group i - 1 go device -> host on a second copy stream (the two directions of the link are independent).
+    HostPipe* hp = host_pipe();
+    if (!hp) return GDN_ERR_CUDA;
+    const Sizes sz = sizes_of(d);
+    auto carve = [&](size_t bytes) -> char* { char* r = ws; ws += round256(bytes); return r; };
+    char* cu_d = carve(sz.cu);
+    char* q_d = carve(sz.qk); char* k_d = carve(sz.qk); char* v_d = carve(sz.v);
+    char* g_d = carve(sz.gb); char* b_d = carve(sz.gb);
+    char* init_d = d->init_state ? carve(sz.state) : nullptr;
+    char* o_d = out_o ? carve(sz.o) : nullptr;
+    char* st_d = out_state ? carve(sz.state) : nullptr;
+    p.cu = (const int32_t*)cu_d; p.q = q_d; p.k = k_d; p.v = v_d; p.g = (const float*)g_d; p.beta = (const float*)b_d;
 
-    cudaError_t e = cudaErrorNotSupported;
-    if (use_tc) {
-        e = gdn::launch_tcgen05(p, sched, stream, &g_last_launches);
-        if (e == cudaErrorNotSupported && d->kernel == GDN_KERNEL_TCGEN05) return GDN_ERR_UNSUPPORTED;
+    // request groups of about equal token counts
+    const int32_t N = d->num_seqs;
+    int32_t bounds[kMaxGroups + 1];
+    int ngroups = 0;
+    {
+        const int want = N < kMaxGroups ? N : kMaxGroups;
+        const int64_t T = d->total_tokens;
+        bounds[0] = 0;
+        for (int gi = 1; gi < want; ++gi) {
+            const int64_t target = T * gi / want;
+            int32_t n = bounds[ngroups];
+            while (n < N && cu[n] < target) ++n;
+            if (n > bounds[ngroups] && n < N) bounds[++ngroups] = n;
+        }
+        bounds[++ngroups] = N;
     }
-    if (e == cudaErrorNotSupported) e = gdn::launch_simt(p, sched, d->io_dtype, stream, &g_last_launches);
-    if (e == cudaErrorNotSupported) return GDN_ERR_UNSUPPORTED;
-    if (e != cudaSuccess) return GDN_ERR_CUDA;
+    const size_t row_qk = (size_t)d->num_qk_heads * d->head_k_dim * io_size(d->io_dtype);
+    const size_t row_v = (size_t)d->num_v_heads * d->head_v_dim * io_size(d->io_dtype);
+    const size_t row_gb = (size_t)d->num_v_heads * sizeof(float);
+    const size_t state1 = (size_t)d->num_v_heads * d->head_k_dim * d->head_v_dim * sizeof(float);
 
-    if (d->memory == GDN_MEM_HOST) {
-        cudaError_t err = cudaSuccess;
-        if (out_o && sz.o) err = cudaMemcpyAsync(out_o, o_stage, sz.o, cudaMemcpyDeviceToHost, stream);
-        if (err == cudaSuccess && out_state && sz.state)
-            err = cudaMemcpyAsync(out_state, st_stage, sz.state, cudaMemcpyDeviceToHost, stream);
-        if (err != cudaSuccess) return GDN_ERR_CUDA;
+    cudaError_t err = cudaEventRecord(hp->ev_start, stream);     // earlier work on the caller's stream (and the last
+    if (err == cudaSuccess) err = cudaStreamWaitEvent(hp->s_in, hp->ev_start, 0);   // call's use of the workspace) first
+    if (err == cudaSuccess) err = cudaStreamWaitEvent(hp->s_out, hp->ev_start, 0);
+    if (err == cudaSuccess) err = cudaMemcpyAsync(cu_d, cu, sz.cu, cudaMemcpyHostToDevice, hp->s_in);
+    auto copy = [&](void* dst, const void* src, size_t bytes, cudaMemcpyKind kind, cudaStream_t st) {
+        if (err == cudaSuccess && bytes) err = cudaMemcpyAsync(dst, src, bytes, kind, st);
+    };
+    int32_t status = GDN_OK;
+    for (int gi = 0; gi < ngroups && err == cudaSuccess && status == GDN_OK; ++gi) {
+        const int32_t n0 = bounds[gi], n1 = bounds[gi + 1];
+        const size_t r0 = (size_t)cu[n0], rows = (size_t)cu[n1] - r0;
+        copy(q_d + r0 * row_qk, (const char*)q + r0 * row_qk, rows * row_qk, cudaMemcpyHostToDevice, hp->s_in);
+        copy(k_d + r0 * row_qk, (const char*)k + r0 * row_qk, rows * row_qk, cudaMemcpyHostToDevice, hp->s_in);
+        copy(v_d + r0 * row_v, (const char*)v + r0 * row_v, rows * row_v, cudaMemcpyHostToDevice, hp->s_in);
+        copy(g_d + r0 * row_gb, (const char*)g + r0 * row_gb, rows * row_gb, cudaMemcpyHostToDevice, hp->s_in);
+        copy(b_d + r0 * row_gb, (const char*)beta + r0 * row_gb, rows * row_gb, cudaMemcpyHostToDevice, hp->s_in);
+        if (init_d)
+            copy(init_d + n0 * state1, (const char*)d->init_state + n0 * state1, (n1 - n0) * state1, cudaMemcpyHostToDevice, hp->s_in);
+        if (err == cudaSuccess) err = cudaEventRecord(hp->ev_in[gi], hp->s_in);
+        if (err == cudaSuccess) err = cudaStreamWaitEvent(stream, hp->ev_in[gi], 0);
+        if (err != cudaSuccess) break;
+        gdn::Problem pg = p;
+        pg.cu = p.cu + n0; pg.num_seqs = n1 - n0;
+        pg.init_state = init_d ? (const float*)(init_d + n0 * state1) : nullptr;
+        pg.out_o = o_d; pg.out_state = st_d ? (float*)(st_d + n0 * state1) : nullptr;
+        gdn::Sched sg = sched;
+        sg.order = sched.order + n0;
+        const int before = g_last_launches;
+        status = run_kernels(pg, sg, use_tc, d->kernel, d->io_dtype, stream);
+        g_last_launches += before;
+        if (status != GDN_OK) break;
+        err = cudaEventRecord(hp->ev_k[gi], stream);
+        if (err == cudaSuccess) err = cudaStreamWaitEvent(hp->s_out, hp->ev_k[gi], 0);
+        if (out_o) copy((char*)out_o + r0 * row_v, o_d + r0 * row_v, rows * row_v, cudaMemcpyDeviceToHost, hp->s_out);
+        if (out_state)
+            copy((char*)out_state + n0 * state1, st_d + n0 * state1, (n1 - n0) * state1, cudaMemcpyDeviceToHost, hp->s_out);
     }
+    // the caller's stream ends the call: it has the results once the last copy back is done
+    cudaError_t e2 = cudaEventRecord(hp->ev_done, hp->s_out);
+    if (e2 == cudaSuccess) e2 = cudaStreamWaitEvent(stream, hp->ev_done, 0);
+    if (status != GDN_OK) return status;
+    if (err != cudaSuccess || e2 != cudaSuccess) return GDN_ERR_CUDA;
     return GDN_OK;
 }
 

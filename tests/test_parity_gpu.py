@@ -309,3 +309,22 @@ def test_randomised_ragged_batches(kernel):
         g_lo, g_hi = decay[it % 4]
         inp = make_inputs(lens, hq, hq * g, 128, 128, "bf16", seed=2608030310 + 50_000 + it, g_lo=g_lo, g_hi=g_hi)
         check(inp, kernel)
+
+
+@pytest.mark.parametrize("kernel", [TC])
+def test_group_parallel_packing_equals_per_layer_calls(kernel):
+    """The paper rebuilds every group independently: the current layer of G groups can therefore go into one call as
+    G pseudo-requests.  The packed call must reproduce the G single-request calls bit for bit (a chain's arithmetic does
+    not depend on what else is in the batch) and match the oracle."""
+    G, L = 12, 410
+    layers = [config_budget_sweep_layer(L, layer=i) for i in range(G)]
+    packed = make_inputs([L] * G, 16, 32, 128, 128, "bf16", seed=1)
+    for name in ("q", "k", "v", "g", "beta", "q_bits", "k_bits", "v_bits"):
+        setattr(packed, name, np.ascontiguousarray(np.concatenate([getattr(x, name) for x in layers], axis=0)))
+    o, st, launches = run_library(packed, kernel=kernel, canary=True)
+    ro, rst = oracle.gdn_forward_inputs(packed)
+    assert_parity(packed, o, st, ro, rst)
+    for i in (0, 5, G - 1):
+        oi, sti, _ = run_library(layers[i], kernel=kernel)
+        np.testing.assert_array_equal(o[i * L:(i + 1) * L], oi)
+        np.testing.assert_array_equal(st[i], sti[0])
