@@ -33,7 +33,7 @@ BASE_SEED = 2608030310
 
 __all__ = [
     "BASE_SEED", "GdnInputs", "f32_to_bf16_bits", "bf16_bits_to_f32",
-    "make_inputs", "tail_lengths_uniform", "config_tiny_f32", "config_single_layer",
+    "make_inputs", "make_raw_inputs", "tail_lengths_uniform", "config_tiny_f32", "config_single_layer",
     "config_budget_sweep_tails", "config_budget_sweep_layer", "config_concurrent_hits", "config_full_prefill",
     "PAPER_PREFIX_LENGTHS", "NOMINAL_PREFIX_LENGTHS", "REPLAY_BUDGETS",
 ]
@@ -166,6 +166,36 @@ def make_inputs(tail_lens: Sequence[int], num_qk_heads: int, num_v_heads: int,
                      num_qk_heads=num_qk_heads, num_v_heads=num_v_heads,
                      head_k_dim=head_k_dim, head_v_dim=head_v_dim, io_dtype=io_dtype,
                      q_bits=qb, k_bits=kb, v_bits=vb, meta=m)
+
+
+def make_raw_inputs(tail_lens: Sequence[int], num_qk_heads: int, num_v_heads: int,
+                    head_k_dim: int, head_v_dim: int, io_dtype: str = "bf16",
+                    seed: int = BASE_SEED, gate_lo: float = 2.2, gate_hi: float = 7.0) -> GdnInputs:
+    """One batch of RAW projection outputs for the fused input stage: q, k ~ N(0, s^2) with a per-token scale
+    s ~ U(0.5, 3) and no normalisation, v ~ N(0,1), the gate pre-activation ~ U(gate_lo, gate_hi) (sigmoid of it
+    in about (0.90, 0.999), the range of the ready-made recipe) and the beta pre-activation ~ N(0,1).  The fields
+    ``q, k, g, beta`` of the result hold these raw values; nothing here applies the input stage."""
+    assert io_dtype in ("bf16", "f32")
+    lens = np.asarray(list(tail_lens), dtype=np.int64)
+    cu = np.zeros(len(lens) + 1, dtype=np.int64)
+    np.cumsum(lens, out=cu[1:])
+    T = int(cu[-1])
+    rng = np.random.Generator(np.random.Philox(key=int(seed) ^ 0x0A57A6E))
+    sq = rng.uniform(0.5, 3.0, size=(T, num_qk_heads, 1)).astype(np.float32)
+    sk = rng.uniform(0.5, 3.0, size=(T, num_qk_heads, 1)).astype(np.float32)
+    q = _normal(rng, (T, num_qk_heads, head_k_dim)) * sq
+    k = _normal(rng, (T, num_qk_heads, head_k_dim)) * sk
+    v = _normal(rng, (T, num_v_heads, head_v_dim))
+    gate = rng.uniform(gate_lo, gate_hi, size=(T, num_v_heads)).astype(np.float32)
+    braw = _normal(rng, (T, num_v_heads))
+    qb = kb = vb = None
+    if io_dtype == "bf16":
+        qb, kb, vb = f32_to_bf16_bits(q), f32_to_bf16_bits(k), f32_to_bf16_bits(v)
+        q, k, v = bf16_bits_to_f32(qb), bf16_bits_to_f32(kb), bf16_bits_to_f32(vb)
+    return GdnInputs(q=q, k=k, v=v, g=gate, beta=braw, cu_tail_lens=cu.astype(np.int32),
+                     num_qk_heads=num_qk_heads, num_v_heads=num_v_heads,
+                     head_k_dim=head_k_dim, head_v_dim=head_v_dim, io_dtype=io_dtype,
+                     q_bits=qb, k_bits=kb, v_bits=vb, meta={"seed": int(seed), "raw": True})
 
 
 def tail_lengths_uniform(num_seqs: int, lo: int, hi: int, seed: int) -> List[int]:

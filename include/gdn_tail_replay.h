@@ -82,6 +82,12 @@ typedef enum {
     GDN_KERNEL_TCGEN05 = 2      /* chunkwise WY form on tcgen05/TMEM; bf16, dk = dv = 128, chunk 64 */
 } gdn_kernel;
 
+/* What the q, k, g and beta arguments of the forward calls hold. */
+typedef enum {
+    GDN_INPUT_READY = 0,        /* q, k as they enter Eq. 1 (normalised by the caller), g = log alpha, beta */
+    GDN_INPUT_RAW = 1           /* raw projection outputs; the kernels apply the input stage themselves, see below */
+} gdn_input_stage;
+
 typedef struct gdn_desc {
     int32_t  num_qk_heads;      /* Hq */
     int32_t  num_v_heads;       /* Hv, a multiple of Hq */
@@ -92,6 +98,8 @@ typedef struct gdn_desc {
     int64_t  total_tokens;      /* T = cu_tail_lens[N]; known to the caller, so no device sync */
     int32_t  memory;            /* gdn_memory */
     int32_t  kernel;            /* gdn_kernel */
+    int32_t  input_stage;       /* gdn_input_stage */
+    int32_t  reserved;          /* 0 */
     const float* init_state;    /* optional [N, Hv, dk, dv] fp32 start state; NULL = zero (Eq. 2) */
     void*    workspace;         /* caller-owned device scratch, 256-byte aligned */
     size_t   workspace_bytes;   /* >= gdn_workspace_size(desc) */
@@ -116,6 +124,18 @@ GDN_API size_t gdn_workspace_size(const gdn_desc* desc);
 GDN_API int32_t gdn_tail_replay(const gdn_desc* desc, const void* q, const void* k, const void* v,
                         const float* g, const float* beta, const int32_t* cu_tail_lens,
                         int32_t chunk, void* out_o, float* out_state);
+
+/*
+ * Fused input stage (desc->input_stage == GDN_INPUT_RAW).  The paper's replay feeds the cached hiddens through the
+ * linear-attention layers, "which produce k, v, T and beta at each replay step" (Method section); it fixes neither
+ * a normalisation nor a gate parametrisation.  With GDN_INPUT_RAW the forward calls take what the projections put
+ * out and apply, in their load path (no extra pass over memory):
+ *     q, k   each row (token, head) L2-normalised:  x / sqrt(sum(x^2) + 1e-6)
+ *     g      holds the gate pre-activation a:       alpha = sigmoid(a),  i.e. log alpha = -log(1 + exp(-a))
+ *     beta   holds the pre-activation b:            beta = sigmoid(b)
+ * v is used as it is.  Available in gdn_tail_replay, gdn_full_prefill and gdn_tail_replay_static_scratch on both
+ * kernel families; gdn_decode_step takes ready-made inputs only.
+ */
 
 /*
  * Full prefill (paper Eq. 1 over the whole matched prefix; the paper's "full" baseline):

@@ -8,6 +8,9 @@ this package; the product never routes through it and shares no code with it.
   (request, v-head) chains only.
 * ``tail_select``  — replay-window arithmetic k = ceil(r * m) (paper, Method section),
   evaluated in exact rational arithmetic.
+* ``prologue``     — the input pipeline in front of the recurrence (L2-normalised q and k,
+  sigmoid gate and beta from raw projection outputs; paper, Method section), plain numpy fp64;
+  ``gdn_forward_f64`` runs the same recurrence on its fp64 results.
 
 Every function is pinned by the CPU tests; none is "parity unpinned".
 """
@@ -47,6 +50,8 @@ def _load():
         ip = ctypes.POINTER(ctypes.c_int32)
         lib.gdn_oracle_forward.restype = ctypes.c_int
         lib.gdn_oracle_forward.argtypes = [fp, fp, fp, fp, fp, ip] + [ctypes.c_int32] * 5 + [dp, dp, dp, ctypes.c_int32]
+        lib.gdn_oracle_forward_f64.restype = ctypes.c_int
+        lib.gdn_oracle_forward_f64.argtypes = [dp, dp, dp, dp, dp, ip] + [ctypes.c_int32] * 5 + [dp, dp, dp, ctypes.c_int32]
         _lib = lib
     return _lib
 
@@ -94,6 +99,57 @@ def gdn_forward(q, k, v, g, beta, cu_tail_lens, init_state: Optional[np.ndarray]
         st.ctypes.data_as(dp), int(threads if threads is not None else default_threads()))
     if rc != 0:
         raise ValueError("gdn_oracle_forward rejected its arguments")
+    return o, st
+
+
+def prologue(q_raw, k_raw, gate_raw, beta_raw, eps: float = 1e-6):
+    """The input pipeline in front of the recurrence (paper, Method section: the cached hiddens are fed through the
+    linear-attention layers, "which produce k, v, T and beta at each replay step"), from raw projection outputs, in
+    fp64.  The paper fixes neither normalisation nor gate parametrisation; the reading taken here:
+
+        q, k   L2-normalised over the head dimension:  x / sqrt(sum(x^2) + eps)
+        alpha  = sigmoid(gate_raw)   so that alpha in (0, 1), i.e.  g = log alpha = -log(1 + exp(-gate_raw))
+        beta   = sigmoid(beta_raw)   in (0, 1)
+
+    Returns (q, k, g, beta) as fp64 arrays."""
+    q = np.asarray(q_raw, dtype=np.float64)
+    k = np.asarray(k_raw, dtype=np.float64)
+    a = np.asarray(gate_raw, dtype=np.float64)
+    b = np.asarray(beta_raw, dtype=np.float64)
+    qn = q / np.sqrt(np.sum(q * q, axis=-1, keepdims=True) + eps)
+    kn = k / np.sqrt(np.sum(k * k, axis=-1, keepdims=True) + eps)
+    g = -np.logaddexp(0.0, -a)
+    beta = 1.0 / (1.0 + np.exp(-b))
+    return qn, kn, g, beta
+
+
+def gdn_forward_f64(q, k, v, g, beta, cu_tail_lens, init_state: Optional[np.ndarray] = None,
+                    threads: Optional[int] = None, want_o: bool = True):
+    """``gdn_forward`` on inputs that are already fp64 (no widening step): same C routine, same recurrence."""
+    lib = _load()
+    q, k, v, g, beta = (np.ascontiguousarray(x, dtype=np.float64) for x in (q, k, v, g, beta))
+    cu = np.ascontiguousarray(cu_tail_lens, dtype=np.int32)
+    T, Hq, dk = q.shape
+    Tv, Hv, dv = v.shape
+    N = cu.shape[0] - 1
+    assert k.shape == q.shape and Tv == T and g.shape == (T, Hv) and beta.shape == (T, Hv)
+    assert cu[0] == 0 and cu[-1] == T
+    o = np.zeros((T, Hv, dv), dtype=np.float64) if want_o else None
+    st = np.zeros((N, Hv, dk, dv), dtype=np.float64)
+    init = None
+    if init_state is not None:
+        init = np.ascontiguousarray(init_state, dtype=np.float64)
+        assert init.shape == st.shape
+    dp = ctypes.POINTER(ctypes.c_double)
+    ip = ctypes.POINTER(ctypes.c_int32)
+    rc = lib.gdn_oracle_forward_f64(
+        q.ctypes.data_as(dp), k.ctypes.data_as(dp), v.ctypes.data_as(dp), g.ctypes.data_as(dp),
+        beta.ctypes.data_as(dp), cu.ctypes.data_as(ip), N, Hq, Hv, dk, dv,
+        init.ctypes.data_as(dp) if init is not None else None,
+        o.ctypes.data_as(dp) if o is not None else None,
+        st.ctypes.data_as(dp), int(threads if threads is not None else default_threads()))
+    if rc != 0:
+        raise ValueError("gdn_oracle_forward_f64 rejected its arguments")
     return o, st
 
 

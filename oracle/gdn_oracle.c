@@ -29,6 +29,7 @@
 
 typedef struct {
     const float *q, *k, *v, *g, *beta;
+    const double *qd, *kd, *vd, *gd, *betad;   /* the same five inputs given in fp64 (then the float ones are NULL) */
     const int32_t *cu;
     int32_t num_seqs, Hq, Hv, dk, dv;
     const double *init_state;
@@ -56,14 +57,14 @@ static void run_chain(const oracle_job *J, int32_t n, int32_t h)
     }
 
     for (int64_t t = J->cu[n]; t < J->cu[n + 1]; ++t) {
-        const double alpha = exp((double)J->g[t * Hv + h]);
-        const double beta = (double)J->beta[t * Hv + h];
+        const double alpha = exp(J->gd ? J->gd[t * Hv + h] : (double)J->g[t * Hv + h]);
+        const double beta = J->betad ? J->betad[t * Hv + h] : (double)J->beta[t * Hv + h];
         for (int32_t j = 0; j < dk; ++j) {
-            kk[j] = (double)J->k[(t * Hq + hq) * dk + j];
-            qq[j] = (double)J->q[(t * Hq + hq) * dk + j];
+            kk[j] = J->kd ? J->kd[(t * Hq + hq) * dk + j] : (double)J->k[(t * Hq + hq) * dk + j];
+            qq[j] = J->qd ? J->qd[(t * Hq + hq) * dk + j] : (double)J->q[(t * Hq + hq) * dk + j];
         }
         for (int32_t i = 0; i < dv; ++i)
-            vv[i] = (double)J->v[(t * Hv + h) * dv + i];
+            vv[i] = J->vd ? J->vd[(t * Hv + h) * dv + i] : (double)J->v[(t * Hv + h) * dv + i];
 
         /* S k  (what the old state recalls for this key) */
         for (int32_t i = 0; i < dv; ++i) {
@@ -110,6 +111,8 @@ static void *worker(void *arg)
     return NULL;
 }
 
+static int run_job(oracle_job *Jp, int32_t num_threads);
+
 /*
  * Returns 0 on success, -1 on bad arguments.  init_state may be NULL (zero start, Eq. 2);
  * out_o or out_state may be NULL to skip that output.  num_threads <= 1 runs inline.
@@ -129,6 +132,31 @@ int gdn_oracle_forward(const float *q, const float *k, const float *v, const flo
     J.q = q; J.k = k; J.v = v; J.g = g; J.beta = beta; J.cu = cu;
     J.num_seqs = num_seqs; J.Hq = Hq; J.Hv = Hv; J.dk = dk; J.dv = dv;
     J.init_state = init_state; J.out_o = out_o; J.out_state = out_state;
+    return run_job(&J, num_threads);
+}
+
+/* The same recurrence on inputs that are already fp64 (what the fp64 input pipeline in front of it produces). */
+int gdn_oracle_forward_f64(const double *q, const double *k, const double *v, const double *g,
+                           const double *beta, const int32_t *cu, int32_t num_seqs, int32_t Hq,
+                           int32_t Hv, int32_t dk, int32_t dv, const double *init_state,
+                           double *out_o, double *out_state, int32_t num_threads)
+{
+    if (!q || !k || !v || !g || !beta || !cu) return -1;
+    if (num_seqs < 0 || Hq <= 0 || Hv <= 0 || Hv % Hq != 0 || dk <= 0 || dv <= 0) return -1;
+    for (int32_t n = 0; n < num_seqs; ++n)
+        if (cu[n + 1] < cu[n]) return -1;
+
+    oracle_job J;
+    memset(&J, 0, sizeof J);
+    J.qd = q; J.kd = k; J.vd = v; J.gd = g; J.betad = beta; J.cu = cu;
+    J.num_seqs = num_seqs; J.Hq = Hq; J.Hv = Hv; J.dk = dk; J.dv = dv;
+    J.init_state = init_state; J.out_o = out_o; J.out_state = out_state;
+    return run_job(&J, num_threads);
+}
+
+static int run_job(oracle_job *Jp, int32_t num_threads)
+{
+    oracle_job J = *Jp;
     J.next_item = 0;
     pthread_mutex_init(&J.lock, NULL);
 

@@ -13,6 +13,7 @@ GDN_OK = 0
 GDN_F32, GDN_BF16 = 0, 1
 GDN_MEM_DEVICE, GDN_MEM_HOST = 0, 1
 GDN_KERNEL_AUTO, GDN_KERNEL_FP32_SIMT, GDN_KERNEL_TCGEN05 = 0, 1, 2
+GDN_INPUT_READY, GDN_INPUT_RAW = 0, 1
 
 
 class GdnError(RuntimeError):
@@ -29,6 +30,7 @@ class GdnDesc(ctypes.Structure):
         ("io_dtype", ctypes.c_int32), ("num_seqs", ctypes.c_int32),
         ("total_tokens", ctypes.c_int64),
         ("memory", ctypes.c_int32), ("kernel", ctypes.c_int32),
+        ("input_stage", ctypes.c_int32), ("reserved", ctypes.c_int32),
         ("init_state", ctypes.c_void_p),
         ("workspace", ctypes.c_void_p), ("workspace_bytes", ctypes.c_size_t),
         ("status_word", ctypes.c_void_p), ("stream", ctypes.c_void_p),
@@ -115,7 +117,7 @@ def _ptr(t) -> Optional[int]:
 
 def _forward(fn_name, q, k, v, g, beta, cu_tail_lens, chunk, out_o, out_state, *, total_tokens=None,
              init_state=None, workspace: Optional[Workspace] = None, status_word=None,
-             kernel: int = GDN_KERNEL_AUTO, stream=None, check: bool = True) -> int:
+             kernel: int = GDN_KERNEL_AUTO, stream=None, check: bool = True, raw_inputs: bool = False) -> int:
     import torch
     lib = load_library()
     host = not q.is_cuda
@@ -148,6 +150,7 @@ def _forward(fn_name, q, k, v, g, beta, cu_tail_lens, chunk, out_o, out_state, *
     desc.total_tokens = T if total_tokens is None else int(total_tokens)
     desc.memory = GDN_MEM_HOST if host else GDN_MEM_DEVICE
     desc.kernel = kernel
+    desc.input_stage = GDN_INPUT_RAW if raw_inputs else GDN_INPUT_READY
     desc.init_state = _ptr(init_state)
     if fn_name == "gdn_tail_replay_static_scratch":
         desc.workspace, desc.workspace_bytes = None, 0          # ignored: the library's built-in scratch is used
@@ -173,7 +176,7 @@ def gdn_tail_replay(q, k, v, g, beta, cu_tail_lens, chunk, out_o, out_state, **k
     All tensors on the GPU (device call) or all on the host (host call: the library stages
     through its workspace and copies results back on the stream).  Asynchronous on the current
     (or given) stream.  Keyword arguments: init_state, workspace, status_word, kernel, stream,
-    check.
+    check, raw_inputs (q, k, g, beta are raw projection outputs: the fused input stage of the header).
     """
     return _forward("gdn_tail_replay", q, k, v, g, beta, cu_tail_lens, chunk, out_o, out_state, **kw)
 

@@ -35,6 +35,7 @@ bool desc_shape_ok(const gdn_desc* d)
     if (d->num_seqs < 0 || d->total_tokens < 0 || d->total_tokens > 0x7fffffffLL) return false;
     if (d->io_dtype != GDN_F32 && d->io_dtype != GDN_BF16) return false;
     if (d->memory != GDN_MEM_DEVICE && d->memory != GDN_MEM_HOST) return false;
+    if (d->input_stage != GDN_INPUT_READY && d->input_stage != GDN_INPUT_RAW) return false;
     if (d->head_k_dim <= 0 || d->head_v_dim <= 0) return false;
     return true;
 }
@@ -150,6 +151,7 @@ int32_t forward(const gdn_desc* d, const void* q, const void* k, const void* v, 
     p.num_seqs = d->num_seqs; p.Hq = d->num_qk_heads; p.Hv = d->num_v_heads;
     p.dk = d->head_k_dim; p.dv = d->head_v_dim; p.total_tokens = d->total_tokens;
     p.status_word = d->status_word;
+    p.input_raw = d->input_stage == GDN_INPUT_RAW ? 1 : 0;
     const bool use_tc = tc_shape && d->kernel != GDN_KERNEL_FP32_SIMT;
 
     if (d->memory == GDN_MEM_DEVICE) {

@@ -20,8 +20,11 @@ struct Problem {
     float* out_state;         // [N, Hv, dk, dv] or nullptr
     int32_t* status_word;     // optional device int32
     int32_t num_seqs, Hq, Hv, dk, dv;
+    int32_t input_raw;        // 1: q, k un-normalised, g = gate pre-activation, beta = pre-activation (fused input stage)
     int64_t total_tokens;
 };
+
+constexpr float kNormEps = 1.0e-6f;   // added to the squared norm of q and k rows in the fused input stage
 
 // Scheduler scratch at the head of the workspace.
 struct SchedHeader {

@@ -91,10 +91,33 @@ gdn_simt_kernel(const Problem p, const Sched s)
             }
             if (tid < kTokBlock) {
                 const bool ok = tid < nvalid;
-                as[tid] = ok ? expf(p.g[(size_t)(row0 + tid) * p.Hv + h]) : 1.f;
-                bs[tid] = ok ? p.beta[(size_t)(row0 + tid) * p.Hv + h] : 0.f;
+                const float gin = ok ? p.g[(size_t)(row0 + tid) * p.Hv + h] : 0.f;
+                const float bin = ok ? p.beta[(size_t)(row0 + tid) * p.Hv + h] : 0.f;
+                if (p.input_raw) {
+                    // fused input stage: alpha = sigmoid(gate), beta = sigmoid(pre-activation)
+                    as[tid] = ok ? 1.f / (1.f + expf(-gin)) : 1.f;
+                    bs[tid] = ok ? 1.f / (1.f + expf(-bin)) : 0.f;
+                } else {
+                    as[tid] = ok ? expf(gin) : 1.f;
+                    bs[tid] = bin;
+                }
             }
             __syncthreads();
+            if (p.input_raw) {
+                // fused input stage: q and k rows L2-normalised, x / sqrt(sum x^2 + eps)
+                for (int t = warp; t < kTokBlock; t += NT / 32) {
+                    float sk = 0.f, sq = 0.f;
+                    for (int d = lane; d < DK; d += 32) { sk = fmaf(ks[t][d], ks[t][d], sk); sq = fmaf(qs[t][d], qs[t][d], sq); }
+#pragma unroll
+                    for (int off = 16; off > 0; off >>= 1) {
+                        sk += __shfl_xor_sync(0xffffffffu, sk, off);
+                        sq += __shfl_xor_sync(0xffffffffu, sq, off);
+                    }
+                    const float rk = rsqrtf(sk + kNormEps), rq = rsqrtf(sq + kNormEps);
+                    for (int d = lane; d < DK; d += 32) { ks[t][d] *= rk; qs[t][d] *= rq; }
+                }
+                __syncthreads();
+            }
             for (int t = warp; t < kTokBlock; t += NT / 32) {
                 float acc = 0.f;
                 for (int d = lane; d < DK; d += 32) acc = fmaf(ks[t][d], qs[t][d], acc);

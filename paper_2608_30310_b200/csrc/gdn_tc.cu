@@ -21,7 +21,7 @@
 //                                              per-token factors; rescaled before c drops below 2^-40)
 //
 // The CTA is warp-specialised and software-pipelined over the chunks of all chains it owns (28 warps):
-//   warp 0       TMA producer: K/Q tiles three chunks ahead (4 slots), V one chunk ahead (1 slot)
+//   warp 0       TMA producer: K/Q tiles two chunks ahead (3 slots), V one chunk ahead (1 slot)
 //   warp 1       issues the chain MMAs (U^T, S0 W^T, the state update, then S0 Q^T and Dl~^T P^T)
 //   warp 2       issues the Gram MMAs, ahead of the chain
 //   warp 3       decay warp: loads g and beta up to three chunks ahead, scans the log-decay and publishes the
@@ -55,9 +55,9 @@ constexpr float kLog2e = 1.4426950408889634f;
 constexpr int kThreads = 896;      // 28 warps, see the role table above (at most 72 registers per thread)
 
 // ---- shared memory map (bytes from a 1024-aligned base) ---------------------------------------
-constexpr uint32_t SM_KQ = 0;                 // 4 slots x {2 halves x [128 rows: K 0-63, Q 64-127] x 128 B} 128 KB
+constexpr uint32_t SM_KQ = 0;                 // 3 slots x {2 halves x [128 rows: K 0-63, Q 64-127] x 128 B}  96 KB
 constexpr uint32_t KQ_SLOT = 32768;
-constexpr uint32_t NKQ = 4;
+constexpr uint32_t NKQ = 3;
 constexpr uint32_t SM_V = SM_KQ + NKQ * KQ_SLOT;   // 2 halves x [64 rows] x 128 B                          16 KB
 constexpr uint32_t SM_WT = SM_V + 16384;      // W^T [dk][t] bf16, 128 rows x 128 B                          16 KB
 constexpr uint32_t SM_TP = SM_WT + 16384;     // 3 x T' [t][s] bf16: A^ from the post-processing, inverted in place  24 KB
@@ -87,11 +87,14 @@ enum Bar {
 //   eG    e^G c_prev         (column factors of T'', so that W^T comes out multiplied by c_prev, as
 //                             S0 = c_prev * stored state; also the output epilogue's factor of (stored state) q)
 //   bRest beta e^(G_C - G) / c   (Delta' = Delta~ diag(bRest) accumulates onto the stored state)
+//   eGk   the column factors of T'' (= eG without the query norms of the fused input stage),  G2p = G2 as the row
+//         decay of P (G2 + log2 of the query row's 1 / norm in the fused input stage)
 //   rescale / wb: this chunk starts from a rescaled state: the previous chunk's state epilogue multiplies the
 //   stored state by wb = c_prev e^(G_C) first;  cfin = c after this chunk (final state = cfin * stored state)
-struct __align__(16) Decay { float G2[64], beta[64], eG[64], bRest[64], colfb[32]; float wb; float G2mid; float cfin; int rescale; int pad[3]; };
+struct __align__(16) Decay { float G2[64], beta[64], eG[64], bRest[64], colfb[32], eGk[64], G2p[64]; float wb; float G2mid; float cfin; int rescale; int pad[3]; };
 static_assert(sizeof(Decay) % 16 == 0, "the decay ring is read with 16-byte vector loads");
 struct Misc {
+    float rk[64];                      // fused input stage: 1 / norm of the chunk's key rows (group G1)
     Decay decay[4];                    // per-chunk decay factors, ring of 4 (decay warp writes; pre and chain read)
     unsigned long long bars[NUM_BARS];
     uint32_t tmem_base;
@@ -449,6 +452,42 @@ __device__ void role_mma_chain(const Ctx& cx, const TcParams& prm)
     }
 }
 
+// Fused input stage, decay warp's part (out of line: ready-made inputs never run it): gate and beta activations of this
+// lane's two tokens, and 1 / norm of their query rows from the Q tile of chunk j (the outputs are linear in q, so the
+// query norms enter as factors of the output rows: in the row decay of P and in the factors of S0 q).
+struct RawIn { float g0, g1, b0, b1, lq0, lq1, rq0, rq1; };
+__device__ __noinline__ RawIn raw_inputs(const Ctx& cx, uint32_t j, int lane, bool ok0, bool ok1, float g0, float g1,
+                                         float b0, float b1)
+{
+    float lq0, lq1, rq0, rq1;
+    // alpha = sigmoid(a): log alpha = -log(1 + e^-a), evaluated as min(a, 0) - log1p(e^-|a|);  beta = sigmoid(b)
+    g0 = ok0 ? fminf(g0, 0.f) - log1pf(__expf(-fabsf(g0))) : 0.f;
+    g1 = ok1 ? fminf(g1, 0.f) - log1pf(__expf(-fabsf(g1))) : 0.f;
+    b0 = ok0 ? 1.f / (1.f + __expf(-b0)) : 0.f;
+    b1 = ok1 ? 1.f / (1.f + __expf(-b1)) : 0.f;
+    cx.wait(B_FULL_KQ0 + j % NKQ, (j / NKQ) & 1u);
+    const uint8_t* qt = cx.sm + SM_KQ + (j % NKQ) * KQ_SLOT + 8192;      // Q rows of the two 64-column halves
+    float s0 = 0.f, s1 = 0.f;
+#pragma unroll 1
+    for (int i = 0; i < 16; ++i) {
+        // 16-byte pieces of the rows in an order that spreads the lanes over the banks (the sum does not care)
+        const uint32_t off = (uint32_t)(i >> 3) * 16384u + (uint32_t)(((i + lane) & 7) << 4);
+        const uint4 x0 = *reinterpret_cast<const uint4*>(qt + off + lane * 128);
+        const uint4 x1 = *reinterpret_cast<const uint4*>(qt + off + (lane + 32) * 128);
+        const uint32_t w0[4] = {x0.x, x0.y, x0.z, x0.w}, w1[4] = {x1.x, x1.y, x1.z, x1.w};
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            s0 = fmaf(bf_lo(w0[e]), bf_lo(w0[e]), s0); s0 = fmaf(bf_hi(w0[e]), bf_hi(w0[e]), s0);
+            s1 = fmaf(bf_lo(w1[e]), bf_lo(w1[e]), s1); s1 = fmaf(bf_hi(w1[e]), bf_hi(w1[e]), s1);
+        }
+    }
+    rq0 = rsqrtf(s0 + kNormEps); rq1 = rsqrtf(s1 + kNormEps);
+    lq0 = __log2f(rq0); lq1 = __log2f(rq1);
+    RawIn r;
+    r.g0 = g0; r.g1 = g1; r.b0 = b0; r.b1 = b1; r.lq0 = lq0; r.lq1 = lq1; r.rq0 = rq0; r.rq1 = rq1;
+    return r;
+}
+
 // ================================================================================================
 // warp 3: decay warp.  Runs up to three chunks ahead of the consumers (ring of four slots), which hides the
 // DRAM latency of the strided g / beta loads.
@@ -464,10 +503,15 @@ __device__ void role_decay(const Ctx& cx, const TcParams& prm)
     for (uint32_t j = 0; cc.valid; ++j, cc.advance()) {
         const int row0 = cc.row0(), nvalid = cc.nvalid(), h = cc.h;
         const bool ok0 = lane < nvalid, ok1 = lane + 32 < nvalid;
-        const float g0 = ok0 ? p.g[(size_t)(row0 + lane) * p.Hv + h] : 0.f;
-        const float g1 = ok1 ? p.g[(size_t)(row0 + lane + 32) * p.Hv + h] : 0.f;
-        const float b0 = ok0 ? p.beta[(size_t)(row0 + lane) * p.Hv + h] : 0.f;
-        const float b1 = ok1 ? p.beta[(size_t)(row0 + lane + 32) * p.Hv + h] : 0.f;
+        float g0 = ok0 ? p.g[(size_t)(row0 + lane) * p.Hv + h] : 0.f;
+        float g1 = ok1 ? p.g[(size_t)(row0 + lane + 32) * p.Hv + h] : 0.f;
+        float b0 = ok0 ? p.beta[(size_t)(row0 + lane) * p.Hv + h] : 0.f;
+        float b1 = ok1 ? p.beta[(size_t)(row0 + lane + 32) * p.Hv + h] : 0.f;
+        float lq0 = 0.f, lq1 = 0.f, rq0 = 1.f, rq1 = 1.f;        // log2 and value of 1 / |q| of this lane's two tokens
+        if (p.input_raw) {
+            const RawIn ri = raw_inputs(cx, j, lane, ok0, ok1, g0, g1, b0, b1);
+            g0 = ri.g0; g1 = ri.g1; b0 = ri.b0; b1 = ri.b1; lq0 = ri.lq0; lq1 = ri.lq1; rq0 = ri.rq0; rq1 = ri.rq1;
+        }
         // clamped so that g = -inf (alpha = 0) keeps every difference of cumulative sums finite; 2^-1e5 is still 0
         float G0 = fmaxf(g0 * kLog2e, -1.0e5f), G1 = fmaxf(g1 * kLog2e, -1.0e5f);
 #pragma unroll
@@ -490,7 +534,9 @@ __device__ void role_decay(const Ctx& cx, const TcParams& prm)
         // decay: every Gam[t, .] of such a row underflows to zero, so its A^ and P rows vanish
         dc.G2[lane] = ok0 ? G0 : -1.0e30f; dc.G2[lane + 32] = ok1 ? G1 : -1.0e30f;
         dc.beta[lane] = b0; dc.beta[lane + 32] = b1;
-        dc.eG[lane] = e0; dc.eG[lane + 32] = e1;
+        dc.eG[lane] = e0 * rq0; dc.eG[lane + 32] = e1 * rq1;
+        dc.eGk[lane] = e0; dc.eGk[lane + 32] = e1;
+        dc.G2p[lane] = ok0 ? G0 + lq0 : -1.0e30f; dc.G2p[lane + 32] = ok1 ? G1 + lq1 : -1.0e30f;
         dc.bRest[lane] = b0 * (ex2_approx(GC - G0) * cinv); dc.bRest[lane + 32] = b1 * (ex2_approx(GC - G1) * cinv);
         const float G31 = __shfl_sync(0xffffffffu, G0, 31);
         dc.colfb[lane] = ex2_approx(G31 - G0) * b0;
@@ -507,6 +553,35 @@ __device__ __noinline__ uint32_t count_chunks(const TcParams& prm)
     uint32_t n = 0;
     while (cc.valid) { n += (uint32_t)cc.nchunks; cc.next_chain(); }
     return n;
+}
+
+// Fused input stage, group G1's part (out of line: ready-made inputs never run it).  The squared norms of the chunk's
+// key rows are the diagonal of K K^T, which sits in the Gram accumulator: one warp per lane window of the K rows reads
+// them, the group meets, 64 of its threads fold 1 / |k_s| into the per-token factors that multiply key s wherever it
+// enters (columns of A^ and P, columns of T'', the state update), the group meets again.  Returns what a row of A^
+// adds to its row decay: log2(1 / |k_t|) (0 for rows of P, whose query norms the decay warp has folded in).
+__device__ __noinline__ float key_norms(const Ctx& cx, Misc* misc, uint32_t c, uint32_t tl, int wtid, int t, bool isA, int hf)
+{
+    Decay& dc = misc->decay[c & 3u];
+    if (isA && hf == 0) {
+        // the diagonal entries of this warp's 32 rows lie in two 16-column blocks (the address is the same for all lanes)
+        uint32_t lo[16], hi[16];
+        tmem_ld16(tl + TM_GRAM + (uint32_t)(t & 32), lo);
+        tmem_ld16(tl + TM_GRAM + (uint32_t)(t & 32) + 16u, hi);
+        tmem_ld_wait();
+        float dg = 0.f;
+#pragma unroll
+        for (int e = 0; e < 16; ++e) dg = ((t & 31) == e) ? __uint_as_float(lo[e]) : ((t & 31) == e + 16) ? __uint_as_float(hi[e]) : dg;
+        misc->rk[t] = rsqrtf(dg + kNormEps);
+    }
+    asm volatile("bar.sync 1, 256;" ::: "memory");
+    if (wtid < 64) {
+        const float r = misc->rk[wtid];
+        dc.beta[wtid] *= r; dc.bRest[wtid] *= r; dc.eGk[wtid] *= r;
+        if (wtid < 32) dc.colfb[wtid] *= r;
+    }
+    asm volatile("bar.sync 1, 256;" ::: "memory");
+    return isA ? __log2f(misc->rk[t]) : 0.f;
 }
 
 // ================================================================================================
@@ -528,7 +603,7 @@ __device__ void role_g1(const Ctx& cx, const TcParams& prm, int wtid)
         // this thread's row of the Gram tile: lane windows 0,1 hold K K^T rows, 2,3 hold Q K^T rows
         const int t = ((w4 & 1) << 5) + lane;
         const bool isA = w4 < 2;
-        const float G2t = dc.G2[t];
+        float G2t = isA ? dc.G2[t] : dc.G2p[t];
         // the solve works on A^ = strict_lower(Gam (K K^T)) diag(beta) (beta on the columns): its inverse P^ gives
         // T' = diag(beta) P^ and T'' = diag(beta) P^ diag(e^G), and the common row factor beta moves into the
         // Delta epilogue, so that P^ itself is one MMA operand and its column-scaled copy the other
@@ -538,6 +613,7 @@ __device__ void role_g1(const Ctx& cx, const TcParams& prm, int wtid)
         const int t_lim = isA ? t : t + 1;                      // keep columns s < t_lim
         cx.wait(B_GRAM_DONE, c & 1u);
         tc_fence_after();
+        if (prm.p.input_raw) G2t += key_norms(cx, misc, c, tl, wtid, t, isA, hf);
         // buffers: P and T' of chunk c were last read by the MMAs of chunk c-3
         if (c >= 3) {
             cx.wait(B_P_FREE0 + c % 3u, ((c / 3u) - 1u) & 1u);
@@ -773,8 +849,8 @@ __device__ void role_g2(const Ctx& cx, const TcParams& prm, int wtid, int team)
 #pragma unroll 1
             for (int ch = 0; ch <= (t >> 3); ++ch) {
                 const uint4 v = *reinterpret_cast<const uint4*>(src + ((ch ^ (t & 7)) << 4));
-                const float4 e0 = *reinterpret_cast<const float4*>(&dc.eG[8 * ch]);
-                const float4 e1 = *reinterpret_cast<const float4*>(&dc.eG[8 * ch + 4]);
+                const float4 e0 = *reinterpret_cast<const float4*>(&dc.eGk[8 * ch]);
+                const float4 e1 = *reinterpret_cast<const float4*>(&dc.eGk[8 * ch + 4]);
                 uint4 o;
                 o.x = mul_bf16x2(v.x, pack_bf16x2(e0.x, e0.y)); o.y = mul_bf16x2(v.y, pack_bf16x2(e0.z, e0.w));
                 o.z = mul_bf16x2(v.z, pack_bf16x2(e1.x, e1.y)); o.w = mul_bf16x2(v.w, pack_bf16x2(e1.z, e1.w));

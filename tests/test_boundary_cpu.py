@@ -37,10 +37,10 @@ def test_header_symbols_are_exported(lib):
 
 
 def test_desc_layout_matches_header():
-    # 6 int32, int64, 2 int32, 2 pointers, size_t, 2 pointers on LP64
-    assert ctypes.sizeof(B.GdnDesc) == 6 * 4 + 8 + 2 * 4 + 8 + 8 + 8 + 8 + 8
-    assert B.GdnDesc.total_tokens.offset == 24 and B.GdnDesc.init_state.offset == 40
-    assert B.GdnDesc.stream.offset == 72
+    # 6 int32, int64, 4 int32, 2 pointers, size_t, 2 pointers on LP64
+    assert ctypes.sizeof(B.GdnDesc) == 6 * 4 + 8 + 4 * 4 + 8 + 8 + 8 + 8 + 8
+    assert B.GdnDesc.total_tokens.offset == 24 and B.GdnDesc.input_stage.offset == 40
+    assert B.GdnDesc.init_state.offset == 48 and B.GdnDesc.stream.offset == 80
 
 
 def test_tail_select_matches_oracle_and_table(lib):

@@ -299,3 +299,45 @@ def test_tail_select_errors():
     assert oracle.tail_select(-1, 0.05) == -1
     assert oracle.tail_select(10, -0.1) == -1
     assert oracle.tail_select(10, float("nan")) == -1
+
+
+# ---- the input stage in front of the recurrence (oracle.prologue) -------------------------------------
+
+def test_prologue_hand_values_and_identities():
+    """3-4-5 triangle, sigmoid symmetry, log-sigmoid at 0 and far out, scale invariance of the normalisation."""
+    q = np.array([[[3.0, 4.0]]]); k = np.array([[[0.0, -2.0]]])
+    a = np.array([[0.0, 40.0, -40.0]]); b = np.array([[0.0, 1.5, -1.5]])
+    qn, kn, g, beta = oracle.prologue(q, k, a, b, eps=0.0)
+    np.testing.assert_allclose(qn, [[[0.6, 0.8]]], rtol=0, atol=1e-15)
+    np.testing.assert_allclose(kn, [[[0.0, -1.0]]], rtol=0, atol=1e-15)
+    np.testing.assert_allclose(g[0, 0], -np.log(2.0), rtol=1e-15)
+    assert abs(g[0, 1]) < 1e-17 and abs(g[0, 2] + 40.0) < 1e-15          # log sigmoid(a): ~0 far right, ~a far left
+    assert beta[0, 0] == 0.5 and abs(beta[0, 1] + beta[0, 2] - 1.0) < 1e-15
+    rng = np.random.default_rng(1)
+    x = rng.standard_normal((5, 3, 16))
+    n1 = oracle.prologue(x, x, np.zeros((5, 2)), np.zeros((5, 2)), eps=0.0)[0]
+    n2 = oracle.prologue(7.5 * x, x, np.zeros((5, 2)), np.zeros((5, 2)), eps=0.0)[0]
+    np.testing.assert_allclose(n1, n2, rtol=1e-14)
+    np.testing.assert_allclose(np.sum(n1 * n1, axis=-1), 1.0, rtol=1e-14)
+    aa = rng.standard_normal((4, 3)) * 3
+    ga = oracle.prologue(x[:4], x[:4], aa, aa)[2]
+    gb = oracle.prologue(x[:4], x[:4], -aa, aa)[2]
+    np.testing.assert_allclose(np.exp(ga) + np.exp(gb), 1.0, rtol=1e-14)  # sigmoid(a) + sigmoid(-a) = 1
+
+
+def test_prologue_composed_with_recurrence_reduces_to_ready_inputs():
+    """Feeding ready-made inputs through the stage changes nothing it should not: unit-norm q, k stay (eps = 0), the
+    logit of alpha gives back g, the logit of beta gives back beta; and the fp64-input entry of the recurrence is the
+    same routine as the fp32-input one (bitwise on fp32-representable values)."""
+    inp = make_inputs([23, 0, 9], 2, 4, 8, 4, "f32", seed=77)
+    alpha = np.exp(inp.g.astype(np.float64)); beta = inp.beta.astype(np.float64)
+    qn, kn, g, b = oracle.prologue(inp.q, inp.k, np.log(alpha / (1 - alpha)), np.log(beta / (1 - beta)), eps=0.0)
+    np.testing.assert_allclose(g, inp.g.astype(np.float64), rtol=1e-9, atol=1e-12)
+    np.testing.assert_allclose(b, beta, rtol=1e-12)
+    o1, s1 = oracle.gdn_forward_inputs(inp)
+    o2, s2 = oracle.gdn_forward_f64(inp.q, inp.k, inp.v, inp.g, inp.beta, inp.cu_tail_lens)
+    np.testing.assert_array_equal(o1, o2)
+    np.testing.assert_array_equal(s1, s2)
+    o3, s3 = oracle.gdn_forward_f64(qn, kn, inp.v, g, b, inp.cu_tail_lens)
+    np.testing.assert_allclose(o3, o1, rtol=0, atol=1e-6)                 # q, k of the recipe are unit rows up to fp32 rounding
+    np.testing.assert_allclose(s3, s1, rtol=0, atol=1e-6)

@@ -6,7 +6,7 @@ import numpy as np
 import pytest
 
 import oracle
-from gdn_workloads import (make_inputs, config_tiny_f32, config_single_layer, config_concurrent_hits,
+from gdn_workloads import (make_inputs, make_raw_inputs, config_tiny_f32, config_single_layer, config_concurrent_hits,
                            config_budget_sweep_tails, config_budget_sweep_layer, config_full_prefill)
 from gpu_utils import run_library, assert_parity, assert_parity_lean, state_rel_fro, TOL
 
@@ -328,3 +328,24 @@ def test_group_parallel_packing_equals_per_layer_calls(kernel):
         oi, sti, _ = run_library(layers[i], kernel=kernel)
         np.testing.assert_array_equal(o[i * L:(i + 1) * L], oi)
         np.testing.assert_array_equal(st[i], sti[0])
+
+
+def _check_raw(inp, kernel):
+    o, st, _ = run_library(inp, kernel=kernel, raw_inputs=True, canary=True)
+    qn, kn, g, beta = oracle.prologue(inp.q, inp.k, inp.g, inp.beta)
+    ro, rst = oracle.gdn_forward_f64(qn, kn, inp.v, g, beta, inp.cu_tail_lens)
+    return assert_parity(inp, o, st, ro, rst)
+
+
+@pytest.mark.parametrize("kernel", [SIMT, TC])
+def test_fused_input_stage_bf16(kernel):
+    """Raw projection outputs in (un-normalised q and k of varying scale, gate and beta pre-activations): the kernels
+    apply the input stage in their load path; the oracle applies its plain fp64 version first."""
+    _check_raw(make_raw_inputs([130, 64, 1, 0, 63, 65, 410, 5], 2, 4, 128, 128, "bf16", seed=61), kernel)
+    _check_raw(make_raw_inputs([700], 1, 2, 128, 128, "bf16", seed=62), kernel)
+    _check_raw(make_raw_inputs([1638], 16, 32, 128, 128, "bf16", seed=63), kernel)
+
+
+def test_fused_input_stage_fp32():
+    _check_raw(make_raw_inputs([150, 0, 1, 64, 65, 17], 2, 4, 64, 64, "f32", seed=64), SIMT)
+    _check_raw(make_raw_inputs([300], 2, 4, 128, 64, "f32", seed=65), 0)
