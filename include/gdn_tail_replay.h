@@ -195,9 +195,10 @@ GDN_API int32_t gdn_tail_replay_static_scratch(const gdn_desc* desc, const void*
 /*
  * Replay-window length k = ceil(budget_frac * prefix_len) (paper, Method section); the
  * window is rows [prefix_len - k, prefix_len).  Clamped to [0, prefix_len]; budget_frac >= 1
- * selects the whole prefix.  A product that is an integer mathematically but lands just above
- * it in binary64 (0.07 * 100) is not rounded up.  Returns -1 if prefix_len < 0,
- * budget_frac < 0 or budget_frac is NaN.  Host-only.
+ * selects the whole prefix.  budget_frac is read as the decimal it was written as (the shortest
+ * decimal that converts to the same double) and the ceiling is taken in integer arithmetic, for
+ * any prefix_len up to 2^63 - 1: 0.07 * 100 gives 7, not the 8 of a binary64 product.  Returns -1
+ * if prefix_len < 0, budget_frac < 0 or budget_frac is NaN.  Host-only.
  */
 GDN_API int64_t tail_select(int64_t prefix_len, double budget_frac);
 

@@ -1,6 +1,8 @@
 // C-ABI entry points: argument validation, workspace carving, host staging and dispatch.
 // Every step of the path itself runs in the kernels of sched.cu, gdn_simt.cu and gdn_tc.cu.
 #include <math.h>
+#include <stdio.h>
+#include <stdlib.h>
 #include <string.h>
 #include <mutex>
 #include "common.cuh"
@@ -326,12 +328,28 @@ int64_t tail_select(int64_t prefix_len, double budget_frac)
 {
     if (prefix_len < 0 || budget_frac != budget_frac || budget_frac < 0.0) return -1;
     if (budget_frac >= 1.0) return prefix_len;
-    const double x = budget_frac * (double)prefix_len;
-    const double eps = 1e-9 * fmax(1.0, x);
-    int64_t k = (int64_t)ceil(x - eps);
-    if (k < 0) k = 0;
-    if (k > prefix_len) k = prefix_len;
-    return k;
+    if (budget_frac == 0.0 || prefix_len == 0) return 0;
+    // The ratio is read as the decimal it was written as: its shortest decimal representation that converts back to
+    // the same binary64, digits x 10^-scale.  The ceiling of prefix_len x digits / 10^scale is then taken in integers,
+    // so that 0.07 x 100 is 7 and no genuine fraction is lost at any size.
+    char buf[40];
+    int prec = 1;
+    for (; prec <= 17; ++prec) {
+        snprintf(buf, sizeof buf, "%.*e", prec - 1, budget_frac);
+        if (strtod(buf, nullptr) == budget_frac) break;
+    }
+    unsigned long long digits = 0;
+    const char* c = buf;
+    for (; *c && *c != 'e'; ++c)
+        if (*c >= '0' && *c <= '9') digits = digits * 10ull + (unsigned long long)(*c - '0');
+    const int exp10 = *c == 'e' ? atoi(c + 1) : 0;           // value = d.ddd x 10^exp10 = digits x 10^(exp10 - (prec - 1))
+    const int scale = (prec - 1) - exp10;                      // > 0 for a ratio below 1
+    const unsigned __int128 num = (unsigned __int128)(unsigned long long)prefix_len * digits;   // < 2^63 x 10^17
+    if (scale > 36) return num > 0 ? 1 : 0;                    // 10^scale exceeds any possible numerator
+    unsigned __int128 den = 1;
+    for (int i = 0; i < scale; ++i) den *= 10u;
+    const unsigned __int128 k = (num + den - 1) / den;
+    return k > (unsigned __int128)(unsigned long long)prefix_len ? prefix_len : (int64_t)k;
 }
 
 const char* gdn_status_string(int32_t status)

@@ -52,6 +52,10 @@ def test_tail_select_matches_oracle_and_table(lib):
     for m in list(range(0, 300)) + [8192, 16384, 32768, 131072, 8225, 16418, 31366, 31847, 10 ** 6]:
         for pct in range(0, 101):
             assert gdn.tail_select(m, pct / 100.0) == oracle.tail_select(m, pct / 100.0), (m, pct)
+    # exact at any size: a genuine fraction is never swallowed, an exact product never rounded up
+    for m in (10 ** 7 + 1, 10 ** 9 + 7, 10 ** 12 + 1, 3 * 10 ** 15 + 11, 2 ** 62 + 1):
+        for r in (0.05, 0.1, 0.07, 0.0333, 1e-9, 0.999999, 1e-300, 0.3):
+            assert gdn.tail_select(m, r) == oracle.tail_select(m, r), (m, r)
     assert gdn.tail_select(-1, 0.1) == -1
     assert gdn.tail_select(5, -0.1) == -1
     assert gdn.tail_select(5, float("nan")) == -1
