@@ -43,7 +43,11 @@
  * aborts or throws.  Problems visible on the host (null pointers, bad head counts,
  * unsupported dims or chunk, workspace too small, misaligned pointers) are reported before
  * any GPU work is enqueued.  Device data (g > 0, NaN, non-monotone cu_tail_lens on the
- * device) is not validated.  A bounded device-side wait that expires writes
+ * device) is not validated.  The tensor-core path reads whole 64-row tiles, so the last tile of
+ * a request covers rows of the request that follows it in the packed arrays: those rows never
+ * influence the result as long as they hold finite values (any magnitude), but an infinity or
+ * a NaN in the first rows of a request can reach the last tile of its predecessor.
+ * A bounded device-side wait that expires writes
  * GDN_ERR_TIMEOUT to *desc->status_word (if given) and the kernel returns early.
  */
 #ifndef GDN_TAIL_REPLAY_H_
