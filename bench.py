@@ -352,6 +352,7 @@ def main():
                     if NCU_TRAFFIC_BYTES_PER_TOKEN_HEAD else None),
         "kernel_ms": kern_ms, "algorithmic_bytes": alg_bytes, "algorithmic_flops": alg_flops,
         "achieved_tflops": alg_flops / (kern_ms * 1e-3) / 1e12, "roofline_ms": max(t_hbm, t_tc) * 1e3,
+        "frac_of_nominal_8000_gbs": achieved_gbs / 8000.0,      # context: the nominal HBM3e figure, not the denominator
     }
 
     # end to end through the same C-ABI call with HOST buffers: pinned inputs copied H2D and

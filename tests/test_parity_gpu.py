@@ -312,6 +312,21 @@ def test_randomised_ragged_batches(kernel):
 
 
 @pytest.mark.parametrize("kernel", [TC])
+def test_many_short_requests(kernel):
+    """2,000 requests of 0-130 tokens (4,000 chains, 27 rounds of the snake schedule over 148 CTAs): almost every chunk is
+    the first and the last of its chain, a quarter of the requests fit no full chunk and some are empty, so the chain
+    switches (start, final-state store, first-chunk shortcuts) are exercised back to back."""
+    rng = np.random.default_rng(2608030310 + 7)
+    lens = [int(x) for x in rng.integers(0, 131, size=2000)]
+    lens[3] = lens[1500] = 0
+    inp = make_inputs(lens, 1, 2, 128, 128, "bf16", seed=2608030310 + 70_000)
+    o, st, launches = run_library(inp, kernel=kernel, canary=True)
+    assert launches == 2                                     # scheduler kernel + forward kernel
+    ro, rst = oracle.gdn_forward_inputs(inp)
+    assert_parity(inp, o, st, ro, rst)
+
+
+@pytest.mark.parametrize("kernel", [TC])
 def test_group_parallel_packing_equals_per_layer_calls(kernel):
     """The paper rebuilds every group independently: the current layer of G groups can therefore go into one call as
     G pseudo-requests.  The packed call must reproduce the G single-request calls bit for bit (a chain's arithmetic does
@@ -344,6 +359,20 @@ def test_fused_input_stage_bf16(kernel):
     _check_raw(make_raw_inputs([130, 64, 1, 0, 63, 65, 410, 5], 2, 4, 128, 128, "bf16", seed=61), kernel)
     _check_raw(make_raw_inputs([700], 1, 2, 128, 128, "bf16", seed=62), kernel)
     _check_raw(make_raw_inputs([1638], 16, 32, 128, 128, "bf16", seed=63), kernel)
+
+
+@pytest.mark.parametrize("kernel", [SIMT, TC])
+def test_fused_input_stage_with_start_state(kernel):
+    """The input stage and a non-zero start state together (a suffix served from raw projection outputs after a
+    replay): the oracle applies its fp64 input stage and starts the recurrence from the same state."""
+    lens = [130, 0, 64, 1, 200]
+    inp = make_raw_inputs(lens, 2, 4, 128, 128, "bf16", seed=66)
+    st0 = np.random.default_rng(66).standard_normal((len(lens), 4, 128, 128)).astype(np.float32)
+    o, st, _ = run_library(inp, kernel=kernel, raw_inputs=True, init_state=st0, canary=True)
+    qn, kn, g, beta = oracle.prologue(inp.q, inp.k, inp.g, inp.beta)
+    ro, rst = oracle.gdn_forward_f64(qn, kn, inp.v, g, beta, inp.cu_tail_lens, init_state=st0.astype(np.float64))
+    assert_parity(inp, o, st, ro, rst)
+    np.testing.assert_array_equal(st[1], st0[1].astype(np.float64))      # the empty request returns its start state
 
 
 def test_fused_input_stage_fp32():
