@@ -66,14 +66,14 @@ int32_t run_kernels(gdn::Problem& p, gdn::Sched sched, bool use_tc, int32_t kern
     g_last_launches = 0;
     // A single request needs no ordering: the tensor-core path then runs without the scheduler kernel, which
     // matters for the batch-1 state rebuild (one call per layer, a few microseconds each).
-    if (use_tc && p.num_seqs == 1 && gdn::tcgen05_supported(p)) {
+    if (use_tc && p.num_seqs == 1 && p.total_tokens > 0 && gdn::tcgen05_supported(p)) {
         sched.order = nullptr;
     } else {
         if (gdn::launch_scheduler(p.cu, p.num_seqs, sched, stream) != cudaSuccess) return GDN_ERR_CUDA;
         g_last_launches += 1;
     }
     cudaError_t e = cudaErrorNotSupported;
-    if (use_tc) {
+    if (use_tc && p.total_tokens > 0) {                       // (a batch of empty requests only gets its states filled in)
         e = gdn::launch_tcgen05(p, sched, stream, &g_last_launches);
         if (e == cudaErrorNotSupported && kernel == GDN_KERNEL_TCGEN05) return GDN_ERR_UNSUPPORTED;
     }
@@ -221,6 +221,9 @@ int32_t forward(const gdn_desc* d, const void* q, const void* k, const void* v, 
         if (err != cudaSuccess) break;
         gdn::Problem pg = p;
         pg.cu = p.cu + n0; pg.num_seqs = n1 - n0;
+        // The rows of later groups are still on their way: the group sees the arrays only up to its own last row, so
+        // that the tile that hangs over the end reads zeros instead of whatever the workspace held before.
+        pg.total_tokens = (int64_t)cu[n1];
         pg.init_state = init_d ? (const float*)(init_d + n0 * state1) : nullptr;
         pg.out_o = o_d; pg.out_state = st_d ? (float*)(st_d + n0 * state1) : nullptr;
         gdn::Sched sg = sched;

@@ -31,7 +31,7 @@ GUARD_BF16 = 0x7BCD                 # bit pattern of the guards (a large finite 
 
 
 def run_library(inp, kernel=0, host=False, fn="gdn_tail_replay", want_o=True, init_state=None,
-                canary=False, raw_inputs=False):
+                canary=False, raw_inputs=False, workspace=None):
     """Returns (o [T,Hv,dv] float64 or None, state [N,Hv,dk,dv] float64, launches).
 
     With ``canary`` the outputs are carved out of larger device buffers whose surrounding guard
@@ -63,7 +63,8 @@ def run_library(inp, kernel=0, host=False, fn="gdn_tail_replay", want_o=True, in
     if init_state is not None:
         init = torch.from_numpy(np.ascontiguousarray(init_state, dtype=np.float32))
         init = init.pin_memory() if host else init.cuda()
-    getattr(gdn, fn)(q, k, v, g, beta, cu, 64, o, st, kernel=kernel, init_state=init, raw_inputs=raw_inputs)
+    getattr(gdn, fn)(q, k, v, g, beta, cu, 64, o, st, kernel=kernel, init_state=init, raw_inputs=raw_inputs,
+                     workspace=workspace)
     torch.cuda.synchronize()
     launches = gdn.last_launch_count()
     if canary:
