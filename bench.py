@@ -383,6 +383,24 @@ def main():
         e2e = {"value": units_all / (te / e2e_steps * 1e-3), "unit": UNIT,
                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps,
                "ms_per_step": te / e2e_steps}
+        # context for the number above: the same input bytes copied host -> device with nothing else on the link
+        # (the floor of any schedule that has to bring the inputs in)
+        if rank == 0:
+            dv_ = torch.empty_like(hv_, device=dev)
+            dq_ = torch.empty_like(hq, device=dev)
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            for rep in range(3):
+                if rep == 1:
+                    a.record(stream)
+                with torch.cuda.stream(stream):
+                    dv_.copy_(hv_, non_blocking=True); dq_.copy_(hq, non_blocking=True); dq_.copy_(hk, non_blocking=True)
+            b.record(stream)
+            torch.cuda.synchronize()
+            cbytes = (hv_.numel() + hq.numel() + hk.numel()) * 2
+            rate = cbytes / (a.elapsed_time(b) / 2 * 1e-3)
+            e2e["h2d_only_gbs"] = rate / 1e9
+            e2e["h2d_only_ms_for_step_inputs"] = h2d / rate * 1e3
+            del dv_, dq_
         del hq, hk, hv_, ho, hs
 
     # us per 32K-hit state rebuild: 36 GDN layers back to back, batch 1, 5 % and 10 % budgets
