@@ -177,16 +177,18 @@ int32_t forward(const gdn_desc* d, const void* q, const void* k, const void* v, 
     char* st_d = out_state ? carve(sz.state) : nullptr;
     p.cu = (const int32_t*)cu_d; p.q = q_d; p.k = k_d; p.v = v_d; p.g = (const float*)g_d; p.beta = (const float*)b_d;
 
-    // request groups of about equal token counts
+    // Request groups by token count.  The link into the device is the busy resource from the first copy to the last, so
+    // what a schedule can save is its tail: the compute and the copy back of the last group.  Six equal groups take
+    // 86 % of the tokens, the last three 8 %, 4 % and 2 %; fewer, larger copies also mean fewer copy launches.
     const int32_t N = d->num_seqs;
     int32_t bounds[kMaxGroups + 1];
     int ngroups = 0;
     {
-        const int want = N < kMaxGroups ? N : kMaxGroups;
+        static const double cum[] = {0.1433, 0.2867, 0.43, 0.5733, 0.7167, 0.86, 0.94, 0.98};
         const int64_t T = d->total_tokens;
         bounds[0] = 0;
-        for (int gi = 1; gi < want; ++gi) {
-            const int64_t target = T * gi / want;
+        for (double f : cum) {
+            const int64_t target = (int64_t)(f * (double)T);
             int32_t n = bounds[ngroups];
             while (n < N && cu[n] < target) ++n;
             if (n > bounds[ngroups] && n < N) bounds[++ngroups] = n;
@@ -195,7 +197,6 @@ int32_t forward(const gdn_desc* d, const void* q, const void* k, const void* v, 
     }
     const size_t row_qk = (size_t)d->num_qk_heads * d->head_k_dim * io_size(d->io_dtype);
     const size_t row_v = (size_t)d->num_v_heads * d->head_v_dim * io_size(d->io_dtype);
-    const size_t row_gb = (size_t)d->num_v_heads * sizeof(float);
     const size_t state1 = (size_t)d->num_v_heads * d->head_k_dim * d->head_v_dim * sizeof(float);
 
     cudaError_t err = cudaEventRecord(hp->ev_start, stream);     // earlier work on the caller's stream (and the last
@@ -205,6 +206,9 @@ int32_t forward(const gdn_desc* d, const void* q, const void* k, const void* v, 
     auto copy = [&](void* dst, const void* src, size_t bytes, cudaMemcpyKind kind, cudaStream_t st) {
         if (err == cudaSuccess && bytes) err = cudaMemcpyAsync(dst, src, bytes, kind, st);
     };
+    // the small per-token arrays go in whole (1 / 64 of the input bytes at d = 128), the large ones group by group
+    copy(g_d, g, sz.gb, cudaMemcpyHostToDevice, hp->s_in);
+    copy(b_d, beta, sz.gb, cudaMemcpyHostToDevice, hp->s_in);
     int32_t status = GDN_OK;
     for (int gi = 0; gi < ngroups && err == cudaSuccess && status == GDN_OK; ++gi) {
         const int32_t n0 = bounds[gi], n1 = bounds[gi + 1];
@@ -212,8 +216,6 @@ int32_t forward(const gdn_desc* d, const void* q, const void* k, const void* v, 
         copy(q_d + r0 * row_qk, (const char*)q + r0 * row_qk, rows * row_qk, cudaMemcpyHostToDevice, hp->s_in);
         copy(k_d + r0 * row_qk, (const char*)k + r0 * row_qk, rows * row_qk, cudaMemcpyHostToDevice, hp->s_in);
         copy(v_d + r0 * row_v, (const char*)v + r0 * row_v, rows * row_v, cudaMemcpyHostToDevice, hp->s_in);
-        copy(g_d + r0 * row_gb, (const char*)g + r0 * row_gb, rows * row_gb, cudaMemcpyHostToDevice, hp->s_in);
-        copy(b_d + r0 * row_gb, (const char*)beta + r0 * row_gb, rows * row_gb, cudaMemcpyHostToDevice, hp->s_in);
         if (init_d)
             copy(init_d + n0 * state1, (const char*)d->init_state + n0 * state1, (n1 - n0) * state1, cudaMemcpyHostToDevice, hp->s_in);
         if (err == cudaSuccess) err = cudaEventRecord(hp->ev_in[gi], hp->s_in);
