@@ -746,6 +746,20 @@ __device__ void role_g2(const Ctx& cx, const TcParams& prm, int wtid, int team)
     const uint32_t mh = cx.sb + SM_MH + team * MH_BYTES;
     const uint32_t J = count_chunks(prm);
     auto pair_sync = [&]() { asm volatile("bar.sync %0, 64;" ::"r"(3 + team) : "memory"); };
+    // The 16-byte pieces of T'' on and below the diagonal (row t has t / 8 + 1 of them, 288 in all) are dealt evenly
+    // to the team's 64 threads, at most 5 each, instead of one row per thread (whose longest rows have 8): ten bits
+    // per piece (row, piece index, valid), fixed for the whole kernel.
+    unsigned long long tpp_items = 0ull;
+    for (int it = 0; it < 5; ++it) {
+        const int i = it * 64 + wtid;
+        if (i < 288) {
+            int g = 0;
+            while (4 * (g + 1) * (g + 2) <= i) ++g;              // rows 8 g .. 8 g + 7 own pieces [4 g (g + 1), 4 (g + 1)(g + 2))
+            const int r = i - 4 * g * (g + 1);
+            const int t = 8 * g + r / (g + 1), ch = r % (g + 1);
+            tpp_items |= (unsigned long long)(512 | (ch << 6) | t) << (10 * it);
+        }
+    }
     // team 0 takes the even chunks, team 1 the odd ones: the A, T' and T'' buffers alternate the same way
 #pragma unroll 1
     for (uint32_t k = (uint32_t)team; k < J; k += 2) {
@@ -839,22 +853,24 @@ __device__ void role_g2(const Ctx& cx, const TcParams& prm, int wtid, int team)
         fence_proxy_async_smem();                               // T' is an MMA operand
         warp_arrive(cx.bar(B_TP_READY0 + k % 3u), lane);
         pair_sync();                                            // the whole inverse is in place
-        // T'' = T' diag(e^G): this thread's row, 16-byte chunks up to the diagonal.  The one T'' buffer was last read by
+        // T'' = T' diag(e^G): this thread's share of the 16-byte pieces up to the diagonal.  The one T'' buffer was last read by
         // the W^T MMA of chunk k-1 (the other team's; consecutive phases of its barrier are observed chunk after chunk).
         if (k >= 1) cx.wait(B_W_DONE0 + ((k - 1) & 1u), ((k - 1) >> 1) & 1u);
         {
-            const int t = 32 * pw + lane;
-            const uint8_t* src = TP + t * 128;
-            uint8_t* dst = cx.sm + SM_TPP + t * 128;
 #pragma unroll 1
-            for (int ch = 0; ch <= (t >> 3); ++ch) {
-                const uint4 v = *reinterpret_cast<const uint4*>(src + ((ch ^ (t & 7)) << 4));
-                const float4 e0 = *reinterpret_cast<const float4*>(&dc.eGk[8 * ch]);
-                const float4 e1 = *reinterpret_cast<const float4*>(&dc.eGk[8 * ch + 4]);
-                uint4 o;
-                o.x = mul_bf16x2(v.x, pack_bf16x2(e0.x, e0.y)); o.y = mul_bf16x2(v.y, pack_bf16x2(e0.z, e0.w));
-                o.z = mul_bf16x2(v.z, pack_bf16x2(e1.x, e1.y)); o.w = mul_bf16x2(v.w, pack_bf16x2(e1.z, e1.w));
-                *reinterpret_cast<uint4*>(dst + ((ch ^ (t & 7)) << 4)) = o;
+            for (int it = 0; it < 5; ++it) {
+                const uint32_t code = (uint32_t)(tpp_items >> (10 * it)) & 1023u;
+                if (code & 512u) {
+                    const int t = (int)(code & 63u), ch = (int)((code >> 6) & 7u);
+                    const uint32_t off = (uint32_t)t * 128u + (uint32_t)((ch ^ (t & 7)) << 4);
+                    const uint4 v = *reinterpret_cast<const uint4*>(TP + off);
+                    const float4 e0 = *reinterpret_cast<const float4*>(&dc.eGk[8 * ch]);
+                    const float4 e1 = *reinterpret_cast<const float4*>(&dc.eGk[8 * ch + 4]);
+                    uint4 o;
+                    o.x = mul_bf16x2(v.x, pack_bf16x2(e0.x, e0.y)); o.y = mul_bf16x2(v.y, pack_bf16x2(e0.z, e0.w));
+                    o.z = mul_bf16x2(v.z, pack_bf16x2(e1.x, e1.y)); o.w = mul_bf16x2(v.w, pack_bf16x2(e1.z, e1.w));
+                    *reinterpret_cast<uint4*>(cx.sm + SM_TPP + off) = o;
+                }
             }
         }
         fence_proxy_async_smem();                               // T'' is an MMA operand
