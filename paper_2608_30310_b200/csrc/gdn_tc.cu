@@ -68,8 +68,8 @@ constexpr uint32_t MH_BYTES = 32 * LDM * 2;   // one per solve team
 constexpr uint32_t SM_MISC = ((SM_MH + 2 * MH_BYTES + 15) / 16) * 16;
 
 enum Bar {
-    B_FULL_KQ0 = 0, B_FULL_KQ1, B_FULL_KQ2, B_FULL_KQ3, B_FULL_V, B_GRAM_DONE, B_W_DONE0, B_W_DONE1, B_U_DONE, B_MMA1_DONE,
-    B_MMA3_DONE, B_STATE_DONE, B_KQ_FREE0, B_KQ_FREE1, B_KQ_FREE2, B_KQ_FREE3, B_P_FREE0, B_P_FREE1, B_P_FREE2,
+    B_FULL_KQ0 = 0, B_FULL_KQ1, B_FULL_KQ2, B_FULL_V, B_GRAM_DONE, B_W_DONE0, B_W_DONE1, B_U_DONE, B_MMA1_DONE,
+    B_MMA3_DONE, B_STATE_DONE, B_KQ_FREE0, B_KQ_FREE1, B_KQ_FREE2, B_P_FREE0, B_P_FREE1, B_P_FREE2,
     B_TP_FREE0, B_TP_FREE1, B_TP_FREE2,
     B_GRAM_READ, B_WACC_READ,
     B_PRE_DONE0, B_PRE_DONE1, B_D_READY, B_SBF_READY, B_ACC23_FREE, B_SQ_DONE,
@@ -78,12 +78,11 @@ enum Bar {
     B_A_READY0, B_A_READY1, B_A_READY2, B_TP_READY0, B_TP_READY1, B_TP_READY2, NUM_BARS
 };
 
-// colf[s] = 2^(G2_31 - G2_s), s < 32: column factors of the purely off-diagonal quadrant of Gam
 // Per-chunk decay factors.  The fp32 state lives in tensor memory divided by a running factor c (the product of
 // the chunk decays since the last rescale), so that a chunk update is a plain accumulation; c is folded into
 // the factors below, and the state is rescaled (c back to 1) before c leaves [2^-40, 1].
 //   G2    log2-domain inclusive cumulative decay,  beta
-//   colf  2^(G2[31] - G2[s]) for s < 32,  colfb = colf * beta[s]
+//   colfb 2^(G2[31] - G2[s]) beta[s] for s < 32: column factors of the purely off-diagonal quadrant of Gam
 //   eG    e^G c_prev         (column factors of T'', so that W^T comes out multiplied by c_prev, as
 //                             S0 = c_prev * stored state; also the output epilogue's factor of (stored state) q)
 //   bRest beta e^(G_C - G) / c   (Delta' = Delta~ diag(bRest) accumulates onto the stored state)
@@ -103,6 +102,7 @@ struct Misc {
 };
 constexpr uint32_t SM_TOTAL = SM_MISC + ((sizeof(Misc) + 15) / 16) * 16;
 constexpr uint32_t SMEM_BYTES = SM_TOTAL + 1008;   // slack for the manual 1024-byte alignment of a 16-byte aligned base
+static_assert(NKQ == 3, "the K/Q barriers are enumerated per slot");
 static_assert(SMEM_BYTES <= 232448, "exceeds the 227 KB shared memory of one CTA");
 
 // ---- TMEM column map (512 columns x 128 lanes x 32 bit) ----------------------------------------
