@@ -249,6 +249,24 @@ def run_sweep(args, dev, gdn):
         r["tokens_heads_per_s"] = m * 32 / (r["us_mean"] * 1e-6)
         out["full_prefill_%d" % m] = r
         del x, oo
+    # the 32-request workload from raw projection outputs (input stage fused into the kernel) and from start states
+    from gdn_workloads import config_concurrent_hits, make_raw_inputs
+    c3 = config_concurrent_hits()
+    lens = [int(b - a) for a, b in zip(c3.cu_tail_lens[:-1], c3.cu_tail_lens[1:])]
+    ready = to_device(c3, dev)
+    raw = to_device(make_raw_inputs(lens, 16, 32, 128, 128, "bf16", seed=2608030310 + 3500), dev)
+    T, N = c3.total_tokens, c3.num_seqs
+    oo = torch.empty((T, 32, 128), dtype=torch.bfloat16, device=dev)
+    ss = torch.empty((N, 32, 128, 128), dtype=torch.float32, device=dev)
+    st0 = torch.randn((N, 32, 128, 128), dtype=torch.float32, device=dev)
+    for name, x, kw in (("ready_inputs", ready, {}), ("raw_inputs_fused_stage", raw, {"raw_inputs": True}),
+                        ("ready_inputs_with_start_states", ready, {"init_state": st0})):
+        def call():
+            gdn.gdn_tail_replay(x[0], x[1], x[2], x[3], x[4], x[5], 64, oo, ss, workspace=ws, kernel=args.kernel,
+                                stream=stream, **kw)
+        r = timed(call)
+        r["tokens_heads_per_s"] = T * 32 / (r["us_mean"] * 1e-6)
+        out["concurrent_hits_32req_" + name] = r
     print(json.dumps({"sweep": out, "unit": "us", "n_gpus": 1, "dtype": "bf16", "data": "synthetic"}), flush=True)
 
 
