@@ -23,7 +23,7 @@
 // The CTA is warp-specialised and software-pipelined over the chunks of all chains it owns (28 warps):
 //   warp 0       TMA producer: K/Q tiles two chunks ahead (3 slots), V one chunk ahead (1 slot)
 //   warp 1       issues the chain MMAs (U^T, S0 W^T, the state update, then S0 Q^T and Dl~^T P^T)
-//   warp 2       issues the Gram MMAs, ahead of the chain
+//   warp 2       issues the Gram MMAs, ahead of the chain (fused input stage: also the query norms of the chunk)
 //   warp 3       decay warp: loads g and beta up to three chunks ahead, scans the log-decay and publishes the
 //                per-chunk decay factors
 //   warps 4-11   group G1 (two warps per TMEM lane window): Gram post-processing of chunk k+1 (A^ straight into the
@@ -75,7 +75,8 @@ enum Bar {
     B_PRE_DONE0, B_PRE_DONE1, B_D_READY, B_SBF_READY, B_ACC23_FREE, B_SQ_DONE,
     B_DECAY_READY0, B_DECAY_READY1, B_DECAY_READY2, B_DECAY_READY3,
     B_DECAY_FREE0, B_DECAY_FREE1, B_DECAY_FREE2, B_DECAY_FREE3,
-    B_A_READY0, B_A_READY1, B_A_READY2, B_TP_READY0, B_TP_READY1, B_TP_READY2, NUM_BARS
+    B_A_READY0, B_A_READY1, B_A_READY2, B_TP_READY0, B_TP_READY1, B_TP_READY2,
+    B_RQ_READY0, B_RQ_READY1, B_RQ_READY2, B_RQ_READY3, NUM_BARS
 };
 
 // Per-chunk decay factors.  The fp32 state lives in tensor memory divided by a running factor c (the product of
@@ -86,11 +87,12 @@ enum Bar {
 //   eG    e^G c_prev         (column factors of T'', so that W^T comes out multiplied by c_prev, as
 //                             S0 = c_prev * stored state; also the output epilogue's factor of (stored state) q)
 //   bRest beta e^(G_C - G) / c   (Delta' = Delta~ diag(bRest) accumulates onto the stored state)
-//   eGk   the column factors of T'' (= eG without the query norms of the fused input stage),  G2p = G2 as the row
-//         decay of P (G2 + log2 of the query row's 1 / norm in the fused input stage)
+//   eGk   the column factors of T'' (= eG; the fused input stage folds the key norms into this copy)
+//   rq    fused input stage only: 1 / norm of the query rows, written by the Gram warp (the outputs are linear in q,
+//         so the query norms multiply the finished output rows)
 //   rescale / wb: this chunk starts from a rescaled state: the previous chunk's state epilogue multiplies the
 //   stored state by wb = c_prev e^(G_C) first;  cfin = c after this chunk (final state = cfin * stored state)
-struct __align__(16) Decay { float G2[64], beta[64], eG[64], bRest[64], colfb[32], eGk[64], G2p[64]; float wb; float G2mid; float cfin; int rescale; int pad[3]; };
+struct __align__(16) Decay { float G2[64], beta[64], eG[64], bRest[64], colfb[32], eGk[64], rq[64]; float wb; float G2mid; float cfin; int rescale; int pad[3]; };
 static_assert(sizeof(Decay) % 16 == 0, "the decay ring is read with 16-byte vector loads");
 struct Misc {
     float rk[64];                      // fused input stage: 1 / norm of the chunk's key rows (group G1)
@@ -137,14 +139,12 @@ struct TcParams {
 struct ChunkCursor {
     const Problem* p;
     const int32_t* order;
-    int r, n, h, hq, row_begin, row_end, nchunks, c;
-    uint32_t num_items;
+    int r, h, hq, row_begin, row_end, nchunks, c;
     bool valid;
 
     __device__ void init(const Problem* pp, const int32_t* ord)
     {
-        p = pp; order = ord; r = -1; c = 0; nchunks = 0; valid = true;
-        num_items = (uint32_t)pp->num_seqs * (uint32_t)pp->Hv;
+        p = pp; order = ord; r = -1;
         next_chain();
     }
     __device__ static uint32_t item_of(int round)
@@ -152,12 +152,28 @@ struct ChunkCursor {
         const uint32_t G = gridDim.x, b = blockIdx.x;
         return (uint32_t)round * G + ((round & 1) ? (G - 1 - b) : b);
     }
-    // Row range and heads of one work item, kept out of line (three integer divisions and two dependent
-    // global loads, needed once per chain by every role): x = first row, y = end row, z = v-head | q/k head << 16,
-    // w = request index.
+    // The next work item of this CTA after round r that has at least one chunk, kept out of line (integer divisions,
+    // dependent global loads and a loop over empty requests, needed once per chain by every role; everything goes and
+    // comes back in registers): x = first row, y = end row, z = v-head | q/k head << 16, w = its round, or -1 when
+    // the CTA's items are exhausted.
+    __device__ __noinline__ static int4 find_chain(const Problem* p, const int32_t* order, int r)
+    {
+        const uint32_t num_items = (uint32_t)p->num_seqs * (uint32_t)p->Hv;
+        for (;;) {
+            ++r;
+            const uint32_t item = item_of(r);
+            if (item >= num_items) return make_int4(0, 0, 0, -1);
+            const int n = order ? order[item / p->Hv] : (int)(item / p->Hv);   // no order list: requests as given
+            const int h = item % p->Hv;
+            const int hq = h / (p->Hv / p->Hq);
+            const int a = p->cu[n], b = p->cu[n + 1];
+            if (b - a > 0) return make_int4(a, b, h | (hq << 16), r);
+        }
+    }
+    // Row range and heads of one work item: x = first row, y = end row, z = v-head | q/k head << 16, w = request index.
     __device__ __noinline__ static int4 lookup(const Problem* p, const int32_t* order, uint32_t item)
     {
-        const int n = order ? order[item / p->Hv] : (int)(item / p->Hv);       // no order list: requests as given
+        const int n = order ? order[item / p->Hv] : (int)(item / p->Hv);
         const int h = item % p->Hv;
         const int hq = h / (p->Hv / p->Hq);
         return make_int4(p->cu[n], p->cu[n + 1], h | (hq << 16), n);
@@ -165,16 +181,12 @@ struct ChunkCursor {
     // moves to the next chain that has at least one chunk
     __device__ void next_chain()
     {
-        for (;;) {
-            ++r;
-            const uint32_t item = item_of(r);
-            if (item >= num_items) { valid = false; return; }
-            const int4 ci = lookup(p, order, item);
-            row_begin = ci.x; row_end = ci.y; h = ci.z & 0xffff; hq = ci.z >> 16; n = ci.w;
-            nchunks = (row_end - row_begin + 63) >> 6;
-            c = 0;
-            if (nchunks > 0) return;
-        }
+        const int4 ci = find_chain(p, order, r);
+        r = ci.w;
+        valid = ci.w >= 0;
+        row_begin = ci.x; row_end = ci.y; h = ci.z & 0xffff; hq = ci.z >> 16;
+        nchunks = (row_end - row_begin + 63) >> 6;
+        c = 0;
     }
     __device__ void advance()
     {
@@ -346,11 +358,44 @@ __device__ void role_producer(const Ctx& cx, const TcParams& prm, const CUtensor
 // advances the start-address field of a shared-memory descriptor by a byte offset
 __device__ __forceinline__ uint64_t desc_add(uint64_t d, uint32_t bytes) { return d + (uint64_t)(bytes >> 4); }
 
+// Fused input stage, Gram warp's part (out of line: ready-made inputs never run it): 1 / norm of the query rows of
+// chunk j from its Q tile, for the output epilogue, which scales the finished output rows with them (the
+// outputs are linear in q).  The warp has just issued the chunk's Gram MMAs and has nothing else to do until the
+// next tiles land, and nothing upstream of the output epilogue waits for these numbers.
+__device__ __noinline__ void query_norms(const Ctx& cx, uint32_t j, int lane)
+{
+    const uint8_t* qt = cx.sm + SM_KQ + (j % NKQ) * KQ_SLOT + 8192;      // Q rows of the two 64-column halves
+    float s0 = 0.f, s1 = 0.f;
+#pragma unroll 1
+    for (int i = 0; i < 16; ++i) {
+        // 16-byte pieces of the rows in an order that spreads the lanes over the banks (the sum does not care)
+        const uint32_t off = (uint32_t)(i >> 3) * 16384u + (uint32_t)(((i + lane) & 7) << 4);
+        const uint4 x0 = *reinterpret_cast<const uint4*>(qt + off + lane * 128);
+        const uint4 x1 = *reinterpret_cast<const uint4*>(qt + off + (lane + 32) * 128);
+        const uint32_t w0[4] = {x0.x, x0.y, x0.z, x0.w}, w1[4] = {x1.x, x1.y, x1.z, x1.w};
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            s0 = fmaf(bf_lo(w0[e]), bf_lo(w0[e]), s0); s0 = fmaf(bf_hi(w0[e]), bf_hi(w0[e]), s0);
+            s1 = fmaf(bf_lo(w1[e]), bf_lo(w1[e]), s1); s1 = fmaf(bf_hi(w1[e]), bf_hi(w1[e]), s1);
+        }
+    }
+    const float rq0 = rsqrtf(s0 + kNormEps), rq1 = rsqrtf(s1 + kNormEps);     // tokens lane and lane + 32
+    // the ring slot is this chunk's once its decay factors are published (the decay warp waits for the slot's last reader)
+    cx.wait(B_DECAY_READY0 + (j & 3u), (j >> 2) & 1u);
+    cx.misc->decay[j & 3u].rq[lane] = rq0;
+    cx.misc->decay[j & 3u].rq[lane + 32] = rq1;
+    warp_arrive(cx.bar(B_RQ_READY0 + (j & 3u)), lane);
+    // the Q tile has been read: second arrival (after the chain's) that releases the K/Q slot in this mode
+    if (lane == 0) mbar_arrive(cx.bar(B_KQ_FREE0 + j % NKQ));
+}
+
 // ================================================================================================
 // warp 2: Gram MMAs.  Gram(j) needs the K/Q tiles of chunk j and the accumulator read by chunk j-1.
 // ================================================================================================
+template <bool RAW>
 __device__ void role_mma_gram(const Ctx& cx, const TcParams& prm)
 {
+    const int lane = threadIdx.x & 31;
     ChunkCursor cc;
     cc.init(&prm.p, prm.s.order);
 #pragma unroll 1
@@ -369,6 +414,7 @@ __device__ void role_mma_gram(const Ctx& cx, const TcParams& prm)
             mma_commit(cx.bar(B_GRAM_DONE));
         }
         __syncwarp();
+        if (RAW) query_norms(cx, j, lane);
     }
 }
 
@@ -452,46 +498,11 @@ __device__ void role_mma_chain(const Ctx& cx, const TcParams& prm)
     }
 }
 
-// Fused input stage, decay warp's part (out of line: ready-made inputs never run it): gate and beta activations of this
-// lane's two tokens, and 1 / norm of their query rows from the Q tile of chunk j (the outputs are linear in q, so the
-// query norms enter as factors of the output rows: in the row decay of P and in the factors of S0 q).
-struct RawIn { float g0, g1, b0, b1, lq0, lq1, rq0, rq1; };
-__device__ __noinline__ RawIn raw_inputs(const Ctx& cx, uint32_t j, int lane, bool ok0, bool ok1, float g0, float g1,
-                                         float b0, float b1)
-{
-    float lq0, lq1, rq0, rq1;
-    // alpha = sigmoid(a): log alpha = -log(1 + e^-a), evaluated as min(a, 0) - log1p(e^-|a|);  beta = sigmoid(b)
-    g0 = ok0 ? fminf(g0, 0.f) - log1pf(__expf(-fabsf(g0))) : 0.f;
-    g1 = ok1 ? fminf(g1, 0.f) - log1pf(__expf(-fabsf(g1))) : 0.f;
-    b0 = ok0 ? 1.f / (1.f + __expf(-b0)) : 0.f;
-    b1 = ok1 ? 1.f / (1.f + __expf(-b1)) : 0.f;
-    cx.wait(B_FULL_KQ0 + j % NKQ, (j / NKQ) & 1u);
-    const uint8_t* qt = cx.sm + SM_KQ + (j % NKQ) * KQ_SLOT + 8192;      // Q rows of the two 64-column halves
-    float s0 = 0.f, s1 = 0.f;
-#pragma unroll 1
-    for (int i = 0; i < 16; ++i) {
-        // 16-byte pieces of the rows in an order that spreads the lanes over the banks (the sum does not care)
-        const uint32_t off = (uint32_t)(i >> 3) * 16384u + (uint32_t)(((i + lane) & 7) << 4);
-        const uint4 x0 = *reinterpret_cast<const uint4*>(qt + off + lane * 128);
-        const uint4 x1 = *reinterpret_cast<const uint4*>(qt + off + (lane + 32) * 128);
-        const uint32_t w0[4] = {x0.x, x0.y, x0.z, x0.w}, w1[4] = {x1.x, x1.y, x1.z, x1.w};
-#pragma unroll
-        for (int e = 0; e < 4; ++e) {
-            s0 = fmaf(bf_lo(w0[e]), bf_lo(w0[e]), s0); s0 = fmaf(bf_hi(w0[e]), bf_hi(w0[e]), s0);
-            s1 = fmaf(bf_lo(w1[e]), bf_lo(w1[e]), s1); s1 = fmaf(bf_hi(w1[e]), bf_hi(w1[e]), s1);
-        }
-    }
-    rq0 = rsqrtf(s0 + kNormEps); rq1 = rsqrtf(s1 + kNormEps);
-    lq0 = __log2f(rq0); lq1 = __log2f(rq1);
-    RawIn r;
-    r.g0 = g0; r.g1 = g1; r.b0 = b0; r.b1 = b1; r.lq0 = lq0; r.lq1 = lq1; r.rq0 = rq0; r.rq1 = rq1;
-    return r;
-}
-
 // ================================================================================================
 // warp 3: decay warp.  Runs up to three chunks ahead of the consumers (ring of four slots), which hides the
 // DRAM latency of the strided g / beta loads.
 // ================================================================================================
+template <bool RAW>
 __device__ void role_decay(const Ctx& cx, const TcParams& prm)
 {
     const Problem& p = prm.p;
@@ -502,15 +513,20 @@ __device__ void role_decay(const Ctx& cx, const TcParams& prm)
 #pragma unroll 1
     for (uint32_t j = 0; cc.valid; ++j, cc.advance()) {
         const int row0 = cc.row0(), nvalid = cc.nvalid(), h = cc.h;
+        const bool first = cc.first();
         const bool ok0 = lane < nvalid, ok1 = lane + 32 < nvalid;
         float g0 = ok0 ? p.g[(size_t)(row0 + lane) * p.Hv + h] : 0.f;
         float g1 = ok1 ? p.g[(size_t)(row0 + lane + 32) * p.Hv + h] : 0.f;
         float b0 = ok0 ? p.beta[(size_t)(row0 + lane) * p.Hv + h] : 0.f;
         float b1 = ok1 ? p.beta[(size_t)(row0 + lane + 32) * p.Hv + h] : 0.f;
-        float lq0 = 0.f, lq1 = 0.f, rq0 = 1.f, rq1 = 1.f;        // log2 and value of 1 / |q| of this lane's two tokens
-        if (p.input_raw) {
-            const RawIn ri = raw_inputs(cx, j, lane, ok0, ok1, g0, g1, b0, b1);
-            g0 = ri.g0; g1 = ri.g1; b0 = ri.b0; b1 = ri.b1; lq0 = ri.lq0; lq1 = ri.lq1; rq0 = ri.rq0; rq1 = ri.rq1;
+        if (RAW) {
+            // fused input stage: alpha = sigmoid(gate), i.e. log alpha = -log(1 + e^-gate) (the gate of a padded row is 0,
+            // its beta is set to 0 below);  beta = sigmoid(b)
+            g0 = -0.6931471805599453f * __log2f(1.f + ex2_approx(-kLog2e * g0));
+            g1 = -0.6931471805599453f * __log2f(1.f + ex2_approx(-kLog2e * g1));
+            b0 = ok0 ? __frcp_rn(1.f + ex2_approx(-kLog2e * b0)) : 0.f;
+            b1 = ok1 ? __frcp_rn(1.f + ex2_approx(-kLog2e * b1)) : 0.f;
+            g0 = ok0 ? g0 : 0.f; g1 = ok1 ? g1 : 0.f;
         }
         // clamped so that g = -inf (alpha = 0) keeps every difference of cumulative sums finite; 2^-1e5 is still 0
         float G0 = fmaxf(g0 * kLog2e, -1.0e5f), G1 = fmaxf(g1 * kLog2e, -1.0e5f);
@@ -521,9 +537,9 @@ __device__ void role_decay(const Ctx& cx, const TcParams& prm)
         }
         G1 += __shfl_sync(0xffffffffu, G0, 31);
         const float GC = __shfl_sync(0xffffffffu, G1, 31);
-        const float cprev = cc.first() ? 1.f : c;
+        const float cprev = first ? 1.f : c;
         const float eGC = ex2_approx(GC);
-        const bool rescale = cc.first() || !(cprev * eGC >= 9.094947e-13f);       // 2^-40; also catches NaN
+        const bool rescale = first || !(cprev * eGC >= 9.094947e-13f);       // 2^-40; also catches NaN
         c = rescale ? 1.f : cprev * eGC;
         const float cinv = rescale ? 1.f : __frcp_rn(c);
         const float e0 = ex2_approx(G0) * cprev, e1 = ex2_approx(G1) * cprev;
@@ -534,9 +550,8 @@ __device__ void role_decay(const Ctx& cx, const TcParams& prm)
         // decay: every Gam[t, .] of such a row underflows to zero, so its A^ and P rows vanish
         dc.G2[lane] = ok0 ? G0 : -1.0e30f; dc.G2[lane + 32] = ok1 ? G1 : -1.0e30f;
         dc.beta[lane] = b0; dc.beta[lane + 32] = b1;
-        dc.eG[lane] = e0 * rq0; dc.eG[lane + 32] = e1 * rq1;
+        dc.eG[lane] = e0; dc.eG[lane + 32] = e1;
         dc.eGk[lane] = e0; dc.eGk[lane + 32] = e1;
-        dc.G2p[lane] = ok0 ? G0 + lq0 : -1.0e30f; dc.G2p[lane + 32] = ok1 ? G1 + lq1 : -1.0e30f;
         dc.bRest[lane] = b0 * (ex2_approx(GC - G0) * cinv); dc.bRest[lane + 32] = b1 * (ex2_approx(GC - G1) * cinv);
         const float G31 = __shfl_sync(0xffffffffu, G0, 31);
         dc.colfb[lane] = ex2_approx(G31 - G0) * b0;
@@ -559,19 +574,27 @@ __device__ __noinline__ uint32_t count_chunks(const TcParams& prm)
 // key rows are the diagonal of K K^T, which sits in the Gram accumulator: one warp per lane window of the K rows reads
 // them, the group meets, 64 of its threads fold 1 / |k_s| into the per-token factors that multiply key s wherever it
 // enters (columns of A^ and P, columns of T'', the state update), the group meets again.  Returns what a row of A^
-// adds to its row decay: log2(1 / |k_t|) (0 for rows of P, whose query norms the decay warp has folded in).
+// adds to its row decay: log2(1 / |k_t|) (0 for rows of P: the query norms multiply the finished output rows instead).
 __device__ __noinline__ float key_norms(const Ctx& cx, Misc* misc, uint32_t c, uint32_t tl, int wtid, int t, bool isA, int hf)
 {
     Decay& dc = misc->decay[c & 3u];
     if (isA && hf == 0) {
-        // the diagonal entries of this warp's 32 rows lie in two 16-column blocks (the address is the same for all lanes)
+        // the diagonal entry of this lane's row lies in the first (lanes 0-15) or second (lanes 16-31) 16-column block of
+        // the warp's rows (the address is the same for all lanes): both are read, then a select tree on the lane bits
         uint32_t lo[16], hi[16];
         tmem_ld16(tl + TM_GRAM + (uint32_t)(t & 32), lo);
         tmem_ld16(tl + TM_GRAM + (uint32_t)(t & 32) + 16u, hi);
         tmem_ld_wait();
-        float dg = 0.f;
+        uint32_t x8[8], x4[4];
 #pragma unroll
-        for (int e = 0; e < 16; ++e) dg = ((t & 31) == e) ? __uint_as_float(lo[e]) : ((t & 31) == e + 16) ? __uint_as_float(hi[e]) : dg;
+        for (int e = 0; e < 8; ++e) {
+            const uint32_t a = (t & 8) ? lo[e + 8] : lo[e], b = (t & 8) ? hi[e + 8] : hi[e];
+            x8[e] = (t & 16) ? b : a;
+        }
+#pragma unroll
+        for (int e = 0; e < 4; ++e) x4[e] = (t & 4) ? x8[e + 4] : x8[e];
+        const uint32_t y0 = (t & 2) ? x4[2] : x4[0], y1 = (t & 2) ? x4[3] : x4[1];
+        const float dg = __uint_as_float((t & 1) ? y1 : y0);
         misc->rk[t] = rsqrtf(dg + kNormEps);
     }
     asm volatile("bar.sync 1, 256;" ::: "memory");
@@ -588,6 +611,7 @@ __device__ __noinline__ float key_norms(const Ctx& cx, Misc* misc, uint32_t c, u
 // warps 4-11: group G1.  Per iteration k: Gram post-processing of chunk k+1 (writes A^ for the solve and the
 // operand P), then the W^T epilogue of chunk k.
 // ================================================================================================
+template <bool RAW>
 __device__ void role_g1(const Ctx& cx, const TcParams& prm, int wtid)
 {
     const int lane = wtid & 31, pw = wtid >> 5;          // pw = 0..7
@@ -603,7 +627,7 @@ __device__ void role_g1(const Ctx& cx, const TcParams& prm, int wtid)
         // this thread's row of the Gram tile: lane windows 0,1 hold K K^T rows, 2,3 hold Q K^T rows
         const int t = ((w4 & 1) << 5) + lane;
         const bool isA = w4 < 2;
-        float G2t = isA ? dc.G2[t] : dc.G2p[t];
+        float G2t = dc.G2[t];
         // the solve works on A^ = strict_lower(Gam (K K^T)) diag(beta) (beta on the columns): its inverse P^ gives
         // T' = diag(beta) P^ and T'' = diag(beta) P^ diag(e^G), and the common row factor beta moves into the
         // Delta epilogue, so that P^ itself is one MMA operand and its column-scaled copy the other
@@ -613,7 +637,7 @@ __device__ void role_g1(const Ctx& cx, const TcParams& prm, int wtid)
         const int t_lim = isA ? t : t + 1;                      // keep columns s < t_lim
         cx.wait(B_GRAM_DONE, c & 1u);
         tc_fence_after();
-        if (prm.p.input_raw) G2t += key_norms(cx, misc, c, tl, wtid, t, isA, hf);
+        if (RAW) G2t += key_norms(cx, misc, c, tl, wtid, t, isA, hf);
         // buffers: P and T' of chunk c were last read by the MMAs of chunk c-3
         if (c >= 3) {
             cx.wait(B_P_FREE0 + c % 3u, ((c / 3u) - 1u) & 1u);
@@ -1034,6 +1058,7 @@ __device__ void role_chain(const Ctx& cx, const TcParams& prm, int wtid)
 // read from the two accumulators as soon as the chunk's last MMAs have completed: first everything is read, combined
 // and rounded into registers, which releases the accumulators for the next chunk early; the stores follow.
 // ================================================================================================
+template <bool RAW>
 __device__ void role_out(const Ctx& cx, const TcParams& prm, int warp, int lane)
 {
     const Problem& p = prm.p;
@@ -1049,6 +1074,7 @@ __device__ void role_out(const Ctx& cx, const TcParams& prm, int warp, int lane)
         const bool first = cc.first() && p.init_state == nullptr;      // zero start state: S0 Q^T was not computed
         const Decay& dc = cx.misc->decay[j & 3u];
         cx.wait(B_DECAY_READY0 + (j & 3u), (j >> 2) & 1u);
+        if (RAW) cx.wait(B_RQ_READY0 + (j & 3u), (j >> 2) & 1u);
         cx.wait(B_MMA3_DONE, j & 1u);
         tc_fence_after();
         // For a fixed token the 128 lanes hold 128 consecutive bf16 of out_o: each warp store writes 64 contiguous bytes
@@ -1077,6 +1103,11 @@ __device__ void role_out(const Ctx& cx, const TcParams& prm, int warp, int lane)
                 if (!first) {
                     o0 = fmaf(eg.x, __uint_as_float(a2[4 * i4]), o0); o1 = fmaf(eg.y, __uint_as_float(a2[4 * i4 + 1]), o1);
                     o2 = fmaf(eg.z, __uint_as_float(a2[4 * i4 + 2]), o2); o3 = fmaf(eg.w, __uint_as_float(a2[4 * i4 + 3]), o3);
+                }
+                if (RAW) {
+                    // fused input stage: the rows are scaled by 1 / norm of their query rows
+                    const float4 rv = *reinterpret_cast<const float4*>(&dc.rq[c0 + 4 * i4]);
+                    o0 *= rv.x; o1 *= rv.y; o2 *= rv.z; o3 *= rv.w;
                 }
                 pk[2 * i4] = pack_bf16x2(o0, o1);
                 pk[2 * i4 + 1] = pack_bf16x2(o2, o3);
@@ -1127,7 +1158,9 @@ gdn_tc_kernel(const TcParams prm, const __grid_constant__ CUtensorMap tm_q,
                                 i == B_A_READY0 || i == B_A_READY1 || i == B_A_READY2;
             const bool out_bar = i == B_ACC23_FREE || (i >= B_DECAY_FREE0 && i <= B_DECAY_FREE3);
             const bool g2_bar = i == B_TP_READY0 || i == B_TP_READY1 || i == B_TP_READY2;
-            mbar_init(cx.bar(i), wg_bar ? 8u : out_bar ? 4u : g2_bar ? 2u : 1u);
+            // (fused input stage: a K/Q slot is released by the chain's last MMAs and by the Gram warp's reading of Q)
+            const bool kq_free2 = prm.p.input_raw && i >= B_KQ_FREE0 && i <= B_KQ_FREE2;
+            mbar_init(cx.bar(i), wg_bar ? 8u : out_bar ? 4u : (g2_bar || kq_free2) ? 2u : 1u);
         }
         fence_mbar_init();
         cx.misc->abort = 0u;
@@ -1144,15 +1177,18 @@ gdn_tc_kernel(const TcParams prm, const __grid_constant__ CUtensorMap tm_q,
     tc_fence_after();
     cx.tmem = cx.misc->tmem_base;
 
+    // the fused input stage is a property of the launch: the roles it touches exist in two versions, and a launch only
+    // ever executes one of them (its instructions never compete for the instruction cache with the other's)
+    const bool fused = prm.p.input_raw != 0;
     if (warp < 4) {
         if (warp == 0) role_producer(cx, prm, &tm_q, &tm_k, &tm_v);
         else if (warp == 1) role_mma_chain(cx, prm);
-        else if (warp == 2) role_mma_gram(cx, prm);
-        else role_decay(cx, prm);
+        else if (warp == 2) { if (fused) role_mma_gram<true>(cx, prm); else role_mma_gram<false>(cx, prm); }
+        else { if (fused) role_decay<true>(cx, prm); else role_decay<false>(cx, prm); }
     } else if (warp >= 24) {
-        role_out(cx, prm, warp, lane);
+        if (fused) role_out<true>(cx, prm, warp, lane); else role_out<false>(cx, prm, warp, lane);
     } else if (warp < 12) {
-        role_g1(cx, prm, tid - 128);
+        if (fused) role_g1<true>(cx, prm, tid - 128); else role_g1<false>(cx, prm, tid - 128);
     } else if (warp < 20) {
         role_chain(cx, prm, tid - 384);
     } else {
