@@ -105,6 +105,7 @@ struct Misc {
 constexpr uint32_t SM_TOTAL = SM_MISC + ((sizeof(Misc) + 15) / 16) * 16;
 constexpr uint32_t SMEM_BYTES = SM_TOTAL + 1008;   // slack for the manual 1024-byte alignment of a 16-byte aligned base
 static_assert(NKQ == 3, "the K/Q barriers are enumerated per slot");
+static_assert(B_FULL_KQ0 == 0 && B_FULL_V == NKQ && NUM_BARS <= 64, "barrier set-up: the producer's four first, one thread each for the rest");
 static_assert(SMEM_BYTES <= 232448, "exceeds the 227 KB shared memory of one CTA");
 
 // ---- TMEM column map (512 columns x 128 lanes x 32 bit) ----------------------------------------
@@ -311,49 +312,60 @@ __device__ __forceinline__ float bf_lo(uint32_t w) { return __uint_as_float(w <<
 __device__ __forceinline__ float bf_hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
 
 // ================================================================================================
-// warp 0: TMA producer
+// warp 0: TMA producer.  Its first tile copies are issued before the CTA-wide start-up barrier (begin), so that they
+// are in flight while tensor memory is allocated, the other barriers are set up and the other roles find their work.
 // ================================================================================================
-__device__ void role_producer(const Ctx& cx, const TcParams& prm, const CUtensorMap* tm_q, const CUtensorMap* tm_k,
-                              const CUtensorMap* tm_v)
-{
+struct Producer {
     ChunkCursor ckq, cv;                 // K/Q runs two chunks ahead of V
-    ckq.init(&prm.p, prm.s.order);
-    cv = ckq;
-    auto load_kq = [&](const ChunkCursor& cc, uint32_t j) {
-        const uint32_t slot = j % NKQ, dst = cx.sb + SM_KQ + slot * KQ_SLOT, bar = cx.bar(B_FULL_KQ0 + slot);
-        if ((int32_t)j == prm.skip_kq_load) return;       // testing aid: this tile never arrives
-        if (elect_one()) {
-            mbar_arrive_expect_tx(bar, 32768u);
-            tma_load_2d(dst, tm_k, cc.hq * 128, cc.row0(), bar);
-            tma_load_2d(dst + 16384, tm_k, cc.hq * 128 + 64, cc.row0(), bar);
-            tma_load_2d(dst + 8192, tm_q, cc.hq * 128, cc.row0(), bar);
-            tma_load_2d(dst + 24576, tm_q, cc.hq * 128 + 64, cc.row0(), bar);
+    uint32_t jkq;
+
+    __device__ void load_kq(const Ctx& cx, const TcParams& prm, const CUtensorMap* tm_q, const CUtensorMap* tm_k)
+    {
+        const uint32_t slot = jkq % NKQ, dst = cx.sb + SM_KQ + slot * KQ_SLOT, bar = cx.bar(B_FULL_KQ0 + slot);
+        if ((int32_t)jkq != prm.skip_kq_load) {           // testing aid: the skipped tile never arrives
+            if (elect_one()) {
+                mbar_arrive_expect_tx(bar, 32768u);
+                tma_load_2d(dst, tm_k, ckq.hq * 128, ckq.row0(), bar);
+                tma_load_2d(dst + 16384, tm_k, ckq.hq * 128 + 64, ckq.row0(), bar);
+                tma_load_2d(dst + 8192, tm_q, ckq.hq * 128, ckq.row0(), bar);
+                tma_load_2d(dst + 24576, tm_q, ckq.hq * 128 + 64, ckq.row0(), bar);
+            }
+            __syncwarp();
         }
-        __syncwarp();
-    };
-    uint32_t jkq = 0;
-    for (; jkq < NKQ - 1 && ckq.valid; ++jkq) { load_kq(ckq, jkq); ckq.advance(); }
+        ckq.advance();
+        ++jkq;
+    }
+    // needs only the barriers of the K/Q slots
+    __device__ void begin(const Ctx& cx, const TcParams& prm, const CUtensorMap* tm_q, const CUtensorMap* tm_k)
+    {
+        ckq.init(&prm.p, prm.s.order);
+        cv = ckq;
+        jkq = 0;
+        while (jkq < NKQ - 1 && ckq.valid) load_kq(cx, prm, tm_q, tm_k);
+    }
+    __device__ void run(const Ctx& cx, const TcParams& prm, const CUtensorMap* tm_q, const CUtensorMap* tm_k,
+                        const CUtensorMap* tm_v)
+    {
 #pragma unroll 1
-    for (uint32_t j = 0; cv.valid && !cx.stop(); ++j) {
-        // V(j): the single slot is free once U^T MMA of chunk j-1 has completed
-        if (j >= 1) cx.wait(B_U_DONE, (j - 1) & 1u);
-        const uint32_t bar = cx.bar(B_FULL_V);
-        if (elect_one()) {
-            mbar_arrive_expect_tx(bar, 16384u);
-            tma_load_2d(cx.sb + SM_V, tm_v, cv.h * 128, cv.row0(), bar);
-            tma_load_2d(cx.sb + SM_V + 8192, tm_v, cv.h * 128 + 64, cv.row0(), bar);
-        }
-        __syncwarp();
-        cv.advance();
-        // K/Q(j+2): its slot held chunk j-1, free once the state-update MMA of chunk j-1 has completed
-        if (ckq.valid) {
-            if (jkq >= NKQ) cx.wait(B_KQ_FREE0 + jkq % NKQ, ((jkq / NKQ) - 1u) & 1u);
-            load_kq(ckq, jkq);
-            ckq.advance();
-            ++jkq;
+        for (uint32_t j = 0; cv.valid && !cx.stop(); ++j) {
+            // V(j): the single slot is free once U^T MMA of chunk j-1 has completed
+            if (j >= 1) cx.wait(B_U_DONE, (j - 1) & 1u);
+            const uint32_t bar = cx.bar(B_FULL_V);
+            if (elect_one()) {
+                mbar_arrive_expect_tx(bar, 16384u);
+                tma_load_2d(cx.sb + SM_V, tm_v, cv.h * 128, cv.row0(), bar);
+                tma_load_2d(cx.sb + SM_V + 8192, tm_v, cv.h * 128 + 64, cv.row0(), bar);
+            }
+            __syncwarp();
+            cv.advance();
+            // K/Q(j+2): its slot held chunk j-1, free once the state-update MMA of chunk j-1 has completed
+            if (ckq.valid) {
+                if (jkq >= NKQ) cx.wait(B_KQ_FREE0 + jkq % NKQ, ((jkq / NKQ) - 1u) & 1u);
+                load_kq(cx, prm, tm_q, tm_k);
+            }
         }
     }
-}
+};
 
 // advances the start-address field of a shared-memory descriptor by a byte offset
 __device__ __forceinline__ uint64_t desc_add(uint64_t d, uint32_t bytes) { return d + (uint64_t)(bytes >> 4); }
@@ -1146,26 +1158,36 @@ gdn_tc_kernel(const TcParams prm, const __grid_constant__ CUtensorMap tm_q,
     cx.misc = reinterpret_cast<Misc*>(cx.sm + SM_MISC);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    Producer prod;
     if (warp == 0) {
+        // the producer's own barriers first, then its first tile copies, then tensor memory
+        if (lane == 0) {
+            prefetch_tmap(&tm_q); prefetch_tmap(&tm_k); prefetch_tmap(&tm_v);
+            for (int i = B_FULL_KQ0; i <= B_FULL_V; ++i) mbar_init(cx.bar(i), 1u);
+            fence_mbar_init();
+            fence_proxy_async_smem();
+        }
+        __syncwarp();
+        prod.begin(cx, prm, &tm_q, &tm_k);
         tmem_alloc(cx.sb + SM_MISC + (uint32_t)offsetof(Misc, tmem_base), 512);
         tmem_relinquish();
-    }
-    if (tid == 32) {
-        for (int i = 0; i < NUM_BARS; ++i) {
-            // arrivals per phase: one per warp of the arriving group (G1 and chain: 8 warps, G2: 2 warps)
-            const bool wg_bar = i == B_GRAM_READ || i == B_D_READY || i == B_SBF_READY ||
-                                i == B_WACC_READ || i == B_PRE_DONE0 || i == B_PRE_DONE1 ||
-                                i == B_A_READY0 || i == B_A_READY1 || i == B_A_READY2;
-            const bool out_bar = i == B_ACC23_FREE || (i >= B_DECAY_FREE0 && i <= B_DECAY_FREE3);
-            const bool g2_bar = i == B_TP_READY0 || i == B_TP_READY1 || i == B_TP_READY2;
-            // (fused input stage: a K/Q slot is released by the chain's last MMAs and by the Gram warp's reading of Q)
-            const bool kq_free2 = prm.p.input_raw && i >= B_KQ_FREE0 && i <= B_KQ_FREE2;
-            mbar_init(cx.bar(i), wg_bar ? 8u : out_bar ? 4u : (g2_bar || kq_free2) ? 2u : 1u);
-        }
+    } else if (tid - 32 > B_FULL_V && tid - 32 < NUM_BARS) {
+        // one thread per barrier.  Arrivals per phase: one per warp of the arriving group (G1 and chain: 8 warps, output
+        // group: 4, a solve team: 2), one for barriers that a single thread or an MMA commit completes; in the fused
+        // input stage a K/Q slot is released by the chain's last MMAs and by the Gram warp's reading of Q
+        const int i = tid - 32;
+        const bool wg_bar = i == B_GRAM_READ || i == B_D_READY || i == B_SBF_READY ||
+                            i == B_WACC_READ || i == B_PRE_DONE0 || i == B_PRE_DONE1 ||
+                            i == B_A_READY0 || i == B_A_READY1 || i == B_A_READY2;
+        const bool out_bar = i == B_ACC23_FREE || (i >= B_DECAY_FREE0 && i <= B_DECAY_FREE3);
+        const bool g2_bar = i == B_TP_READY0 || i == B_TP_READY1 || i == B_TP_READY2;
+        const bool kq_free2 = prm.p.input_raw && i >= B_KQ_FREE0 && i <= B_KQ_FREE2;
+        mbar_init(cx.bar(i), wg_bar ? 8u : out_bar ? 4u : (g2_bar || kq_free2) ? 2u : 1u);
         fence_mbar_init();
-        cx.misc->abort = 0u;
-        cx.misc->timeout_ns = prm.wait_timeout_ns;
-        prefetch_tmap(&tm_q); prefetch_tmap(&tm_k); prefetch_tmap(&tm_v);
+        if (i == NUM_BARS - 1) {
+            cx.misc->abort = 0u;
+            cx.misc->timeout_ns = prm.wait_timeout_ns;
+        }
     }
     // the operand tiles T' (3), T'' and P (3), contiguous, are only ever written on and below their 16 x 16 diagonal
     // blocks: everything else is zeroed once, here
@@ -1181,7 +1203,7 @@ gdn_tc_kernel(const TcParams prm, const __grid_constant__ CUtensorMap tm_q,
     // ever executes one of them (its instructions never compete for the instruction cache with the other's)
     const bool fused = prm.p.input_raw != 0;
     if (warp < 4) {
-        if (warp == 0) role_producer(cx, prm, &tm_q, &tm_k, &tm_v);
+        if (warp == 0) prod.run(cx, prm, &tm_q, &tm_k, &tm_v);
         else if (warp == 1) role_mma_chain(cx, prm);
         else if (warp == 2) { if (fused) role_mma_gram<true>(cx, prm); else role_mma_gram<false>(cx, prm); }
         else { if (fused) role_decay<true>(cx, prm); else role_decay<false>(cx, prm); }
