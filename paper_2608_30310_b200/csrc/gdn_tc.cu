@@ -1158,9 +1158,16 @@ gdn_tc_kernel(const TcParams prm, const __grid_constant__ CUtensorMap tm_q,
     cx.misc = reinterpret_cast<Misc*>(cx.sm + SM_MISC);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    // Start-up.  Everybody zeroes its share of the operand tiles T' (3), T'' and P (3), contiguous, which are only ever
+    // written on and below their 16 x 16 diagonal blocks.  The producer then sets up the barriers of its own slots and
+    // goes straight to its first tile copies; it only announces itself at the start-up barrier (named barrier 2) and
+    // joins the others again (named barrier 5) before its main loop, which needs their barriers.  Warp 3 allocates
+    // tensor memory, threads 36.. set up one barrier each.
+    for (uint32_t i = tid; i < 7u * 8192u / 16u; i += kThreads)
+        *reinterpret_cast<uint4*>(cx.sm + SM_TP + i * 16u) = make_uint4(0u, 0u, 0u, 0u);
+    fence_proxy_async_smem();
     Producer prod;
     if (warp == 0) {
-        // the producer's own barriers first, then its first tile copies, then tensor memory
         if (lane == 0) {
             prefetch_tmap(&tm_q); prefetch_tmap(&tm_k); prefetch_tmap(&tm_v);
             for (int i = B_FULL_KQ0; i <= B_FULL_V; ++i) mbar_init(cx.bar(i), 1u);
@@ -1168,35 +1175,36 @@ gdn_tc_kernel(const TcParams prm, const __grid_constant__ CUtensorMap tm_q,
             fence_proxy_async_smem();
         }
         __syncwarp();
+        asm volatile("bar.arrive 2, %0;" ::"n"(kThreads) : "memory");
         prod.begin(cx, prm, &tm_q, &tm_k);
-        tmem_alloc(cx.sb + SM_MISC + (uint32_t)offsetof(Misc, tmem_base), 512);
-        tmem_relinquish();
-    } else if (tid - 32 > B_FULL_V && tid - 32 < NUM_BARS) {
-        // one thread per barrier.  Arrivals per phase: one per warp of the arriving group (G1 and chain: 8 warps, output
-        // group: 4, a solve team: 2), one for barriers that a single thread or an MMA commit completes; in the fused
-        // input stage a K/Q slot is released by the chain's last MMAs and by the Gram warp's reading of Q
-        const int i = tid - 32;
-        const bool wg_bar = i == B_GRAM_READ || i == B_D_READY || i == B_SBF_READY ||
-                            i == B_WACC_READ || i == B_PRE_DONE0 || i == B_PRE_DONE1 ||
-                            i == B_A_READY0 || i == B_A_READY1 || i == B_A_READY2;
-        const bool out_bar = i == B_ACC23_FREE || (i >= B_DECAY_FREE0 && i <= B_DECAY_FREE3);
-        const bool g2_bar = i == B_TP_READY0 || i == B_TP_READY1 || i == B_TP_READY2;
-        const bool kq_free2 = prm.p.input_raw && i >= B_KQ_FREE0 && i <= B_KQ_FREE2;
-        mbar_init(cx.bar(i), wg_bar ? 8u : out_bar ? 4u : (g2_bar || kq_free2) ? 2u : 1u);
-        fence_mbar_init();
-        if (i == NUM_BARS - 1) {
-            cx.misc->abort = 0u;
-            cx.misc->timeout_ns = prm.wait_timeout_ns;
+        asm volatile("bar.sync 5, %0;" ::"n"(kThreads) : "memory");
+    } else {
+        if (warp == 3) {
+            tmem_alloc(cx.sb + SM_MISC + (uint32_t)offsetof(Misc, tmem_base), 512);
+            tmem_relinquish();
+        } else if (tid - 32 > B_FULL_V && tid - 32 < NUM_BARS) {
+            // Arrivals per phase: one per warp of the arriving group (G1 and chain: 8 warps, output group: 4, a solve
+            // team: 2), one for barriers that a single thread or an MMA commit completes; in the fused input stage a
+            // K/Q slot is released by the chain's last MMAs and by the Gram warp's reading of Q
+            const int i = tid - 32;
+            const bool wg_bar = i == B_GRAM_READ || i == B_D_READY || i == B_SBF_READY ||
+                                i == B_WACC_READ || i == B_PRE_DONE0 || i == B_PRE_DONE1 ||
+                                i == B_A_READY0 || i == B_A_READY1 || i == B_A_READY2;
+            const bool out_bar = i == B_ACC23_FREE || (i >= B_DECAY_FREE0 && i <= B_DECAY_FREE3);
+            const bool g2_bar = i == B_TP_READY0 || i == B_TP_READY1 || i == B_TP_READY2;
+            const bool kq_free2 = prm.p.input_raw && i >= B_KQ_FREE0 && i <= B_KQ_FREE2;
+            mbar_init(cx.bar(i), wg_bar ? 8u : out_bar ? 4u : (g2_bar || kq_free2) ? 2u : 1u);
+            fence_mbar_init();
+            if (i == NUM_BARS - 1) {
+                cx.misc->abort = 0u;
+                cx.misc->timeout_ns = prm.wait_timeout_ns;
+            }
         }
+        tc_fence_before();
+        asm volatile("bar.sync 2, %0;" ::"n"(kThreads) : "memory");
+        asm volatile("bar.arrive 5, %0;" ::"n"(kThreads) : "memory");
+        tc_fence_after();
     }
-    // the operand tiles T' (3), T'' and P (3), contiguous, are only ever written on and below their 16 x 16 diagonal
-    // blocks: everything else is zeroed once, here
-    for (uint32_t i = tid; i < 7u * 8192u / 16u; i += kThreads)
-        *reinterpret_cast<uint4*>(cx.sm + SM_TP + i * 16u) = make_uint4(0u, 0u, 0u, 0u);
-    fence_proxy_async_smem();
-    tc_fence_before();
-    __syncthreads();
-    tc_fence_after();
     cx.tmem = cx.misc->tmem_base;
 
     // the fused input stage is a property of the launch: the roles it touches exist in two versions, and a launch only
@@ -1225,7 +1233,7 @@ gdn_tc_kernel(const TcParams prm, const __grid_constant__ CUtensorMap tm_q,
         if (tid == 0 && prm.p.status_word) *prm.p.status_word = GDN_ERR_TIMEOUT;
         __syncthreads();
     }
-    if (warp == 0) tmem_dealloc(cx.tmem, 512);
+    if (warp == 3) tmem_dealloc(cx.tmem, 512);
 }
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
