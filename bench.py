@@ -33,9 +33,9 @@ BYTES_PER_TOKEN_HEAD = 776.0        # q,k shared by 2 v-heads + v + o in bf16, g
 FLOPS_PER_TOKEN_HEAD = 139264.0     # 6 dk dv + C (3 dk + 2 dv), triangular products at half cost
 STATE_BYTES_PER_CHAIN = 128 * 128 * 4
 # DRAM bytes per token*head of the dominant kernel, from the committed ncu capture of the 8-request case
-# (profiles/gdn_tc_kernel_concurrent_hits_8req.md: dram read + write = 277.4 MB for 346,944 token*heads,
+# (profiles/gdn_tc_kernel_concurrent_hits_8req.md: dram read + write = 278.2 MB for 346,944 token*heads,
 # final states included); traffic grows in proportion to the units a launch processes.
-NCU_TRAFFIC_BYTES_PER_TOKEN_HEAD = 799.5
+NCU_TRAFFIC_BYTES_PER_TOKEN_HEAD = 801.8
 
 
 def load_peaks():
