@@ -370,11 +370,11 @@ struct Producer {
 // advances the start-address field of a shared-memory descriptor by a byte offset
 __device__ __forceinline__ uint64_t desc_add(uint64_t d, uint32_t bytes) { return d + (uint64_t)(bytes >> 4); }
 
-// Fused input stage, Gram warp's part (out of line: ready-made inputs never run it): 1 / norm of the query rows of
+// Fused input stage, Gram warp's part (inlined into the warp's fused-stage instance only): 1 / norm of the query rows of
 // chunk j from its Q tile, for the output epilogue, which scales the finished output rows with them (the
 // outputs are linear in q).  The warp has just issued the chunk's Gram MMAs and has nothing else to do until the
 // next tiles land, and nothing upstream of the output epilogue waits for these numbers.
-__device__ __noinline__ void query_norms(const Ctx& cx, uint32_t j, int lane)
+__device__ __forceinline__ void query_norms(const Ctx& cx, uint32_t j, int lane)
 {
     const uint8_t* qt = cx.sm + SM_KQ + (j % NKQ) * KQ_SLOT + 8192;      // Q rows of the two 64-column halves
     float s0 = 0.f, s1 = 0.f;
@@ -582,12 +582,12 @@ __device__ __noinline__ uint32_t count_chunks(const TcParams& prm)
     return n;
 }
 
-// Fused input stage, group G1's part (out of line: ready-made inputs never run it).  The squared norms of the chunk's
+// Fused input stage, group G1's part (inlined into the group's fused-stage instance only).  The squared norms of the chunk's
 // key rows are the diagonal of K K^T, which sits in the Gram accumulator: one warp per lane window of the K rows reads
 // them, the group meets, 64 of its threads fold 1 / |k_s| into the per-token factors that multiply key s wherever it
 // enters (columns of A^ and P, columns of T'', the state update), the group meets again.  Returns what a row of A^
 // adds to its row decay: log2(1 / |k_t|) (0 for rows of P: the query norms multiply the finished output rows instead).
-__device__ __noinline__ float key_norms(const Ctx& cx, Misc* misc, uint32_t c, uint32_t tl, int wtid, int t, bool isA, int hf)
+__device__ __forceinline__ float key_norms(const Ctx& cx, Misc* misc, uint32_t c, uint32_t tl, int wtid, int t, bool isA, int hf)
 {
     Decay& dc = misc->decay[c & 3u];
     if (isA && hf == 0) {
